@@ -1,0 +1,240 @@
+"""Pins for the CPU oracle's search part (no GPU).
+
+Each test fixes the oracle against something other than itself: the plain
+definition (exhaustive enumeration), hand-derived values, closed forms,
+textbook special cases computed by a library routine, and invariants.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import scipy.sparse as sp
+from scipy.sparse.csgraph import dijkstra
+
+from paper_2504_03662_b200 import inputs
+
+INF = 2 ** 30 - 1
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def numpy_enumerate(time, mem, trans, budget):
+    """Definition of the problem in itertools (independent of the C enumerator)."""
+    L, S = time.shape
+    best = None
+    for p in itertools.product(range(S), repeat=L):
+        if sum(int(mem[l, p[l]]) for l in range(L)) > budget:
+            continue
+        c = sum(int(time[l, p[l]]) for l in range(L)) + sum(int(trans[p[l - 1], p[l]]) for l in range(1, L))
+        key = (c, tuple(reversed(p)))
+        if best is None or key < best[0]:
+            best = (key, p)
+    return (INF, None) if best is None else (best[0][0], list(best[1]))
+
+
+def test_splitmix64_published_vectors():
+    # First outputs of splitmix64 for state 0 are the published test vector of the generator.
+    assert [int(v) for v in inputs.splitmix64(0, 3)] == [0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4, 0x06C45D188009454F]
+    # skip= gives the same stream
+    assert (inputs.splitmix64(7, 5, skip=3) == inputs.splitmix64(7, 8)[3:]).all()
+
+
+def test_hand_worked_example(orc):
+    # L=2, S=2, M=3.  By hand:
+    #  layer 0: C[0][m] = [5 if m>=1, 3 if m>=2]
+    #  C[1][3][0]: m'=3-2=1 -> prev [5,inf]: 5+trans[0][0]=5 -> +4 = 9 (arg 0)
+    #  C[1][3][1]: m'=3-1=2 -> prev [5,3]:  min(5+2, 3+0)=3 -> +6 = 9 (arg 1)
+    #  tie on the last layer -> strategy 0 -> plan [0,0], memory 1+2=3
+    #  budget 2: C[1][2] = [inf, 5+2+6=13] -> plan [0,1]; budget 1: infeasible
+    time = np.array([[5, 3], [4, 6]]); mem = np.array([[1, 2], [2, 1]]); trans = np.array([[0, 2], [1, 0]])
+    Ct, At = orc.dp(time, mem, trans, 3)
+    assert Ct[0].tolist() == [[INF, INF], [5, INF], [5, 3], [5, 3]]
+    assert Ct[1][3].tolist() == [9, 9] and At[1][3].tolist() == [0, 1]
+    assert Ct[1][2].tolist() == [INF, 13] and At[1][2].tolist() == [255, 0]
+    assert Ct[1][1].tolist() == [INF, INF]
+    for A in (None, At):
+        opt, plan, used, st = orc.backtrack(time, mem, trans, Ct, A, 3)
+        assert (opt, plan.tolist(), used, st) == (9, [0, 0], 3, 0)
+        opt, plan, used, st = orc.backtrack(time, mem, trans, Ct, A, 2)
+        assert (opt, plan.tolist(), used, st) == (13, [0, 1], 2, 0)
+        opt, plan, used, st = orc.backtrack(time, mem, trans, Ct, A, 1)
+        assert (opt, plan.tolist(), st) == (INF, [-1, -1], orc.INFEASIBLE)
+
+
+def test_tie_order_is_last_layer_first(orc):
+    # Plans [1,0] and [0,1] both cost 10; ordered by (p_1, p_0) the first is (0,1) -> plan [1,0].
+    time = np.array([[4, 5], [5, 6]]); mem = np.zeros((2, 2), int); trans = np.array([[9, 0], [0, 9]])
+    # costs: [0,0]=4+5+9=18, [0,1]=4+6+0=10, [1,0]=5+5+0=10, [1,1]=5+6+9=20
+    opt, plan, used, n = orc.brute_force(time, mem, trans, 0)
+    assert (opt, plan.tolist(), n) == (10, [1, 0], 4)
+    r = orc.search(time, mem, trans, 0)
+    assert r["opt_cost"] == 10 and r["plan"].tolist() == [1, 0]
+    assert numpy_enumerate(time, mem, trans, 0) == (10, [1, 0])
+
+
+def test_config0_against_exhaustive_golden(orc):
+    w = inputs.config0()
+    t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
+    Ct, At = orc.dp(t, m, x, w.M)
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "config0_bruteforce.txt")) if not l.startswith("#")]
+    assert len(rows) == w.M + 1
+    for r in rows:
+        budget, opt, used = int(r[0]), int(r[1]), int(r[2])
+        plan = [int(v) for v in r[4:]]
+        for A in (None, At):
+            o, p, u, st = orc.backtrack(t, m, x, Ct, A, budget)
+            assert (o, p.tolist()) == (opt, plan), budget
+            if opt < INF:
+                assert u == used and st == 0
+            else:
+                assert st == orc.INFEASIBLE
+    # the C enumerator agrees with an itertools enumeration at a few budgets
+    for budget in (17, 18, 20, 30, 64):
+        o, p, _, _ = orc.brute_force(t, m, x, budget)
+        eo, ep = numpy_enumerate(t, m, x, budget)
+        assert o == eo and (ep is None or p.tolist() == ep)
+    assert 1296 == 6 ** 4 and int(rows[-1][3]) == 1231   # feasible plans at the full budget
+
+
+@pytest.mark.parametrize("seed", range(240))
+def test_random_tiny_against_exhaustive(orc, seed):
+    rng = np.random.default_rng(seed)
+    L, S, M = int(rng.integers(1, 7)), int(rng.integers(1, 6)), int(rng.integers(0, 41))
+    mode = seed % 4
+    w = inputs.random_tables(1000 + seed, 1, L, S, M, time_hi=(6 if mode == 1 else 10000),
+                             mem_lo=(0 if mode != 2 else 1), mem_hi=max(1, (M // 2 if mode == 3 else M // 3) + (mode == 2) * M),
+                             trans_hi=(3 if mode == 1 else 2000), dup_cols=(mode == 1))
+    t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
+    Ct, At = orc.dp(t, m, x, M)
+    for budget in sorted({0, M // 3, M // 2, M}):
+        eo, ep, eu, _ = orc.brute_force(t, m, x, budget)
+        for A in (None, At):
+            o, p, u, st = orc.backtrack(t, m, x, Ct, A, budget)
+            assert o == eo and p.tolist() == ep.tolist()
+            if eo < INF:
+                assert u == eu <= budget and orc.plan_cost(t, m, x, p) == (o, u)
+    if seed % 16 == 0:
+        eo, ep = numpy_enumerate(t, m, x, M)
+        o, p, _, _ = orc.brute_force(t, m, x, M)
+        assert o == eo and (ep is None or p.tolist() == ep)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_invariants(orc, seed):
+    w = inputs.random_tables(50 + seed, 1, 9, 7, 150, mem_lo=0, mem_hi=40, dup_cols=(seed % 2 == 0))
+    t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
+    Ct, At = orc.dp(t, m, x, w.M)
+    # non-increasing in the budget
+    assert (Ct[:, :-1, :] >= Ct[:, 1:, :]).all()
+    # infeasible below the cheapest possible memory of layers 0..l ending in s
+    lo = np.cumsum(m.min(axis=1)) - m.min(axis=1)
+    for l in range(9):
+        for s in range(7):
+            need = lo[l] + m[l, s]
+            assert (Ct[l, :need, s] == INF).all()
+            assert (Ct[l, need:, s] < INF).all()      # and feasible from there on
+    assert ((At == 255) == (np.concatenate([np.ones_like(Ct[:1], bool), Ct[1:] == INF]))).all()
+    for budget in (0, 30, 77, 150):
+        o, p, u, st = orc.backtrack(t, m, x, Ct, None, budget)
+        o2, p2, u2, st2 = orc.backtrack(t, m, x, Ct, At, budget)
+        assert (o, p.tolist(), u, st) == (o2, p2.tolist(), u2, st2)
+        if o < INF:
+            assert orc.plan_cost(t, m, x, p) == (o, u) and u <= budget
+            assert o == Ct[-1, budget].min() and p[-1] == int(Ct[-1, budget].argmin())
+
+
+def test_single_strategy_closed_form(orc):
+    w = inputs.random_tables(5, 1, 12, 1, 200, mem_lo=3, mem_hi=30)
+    t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
+    x[:] = 777           # never used between equal strategies? it is: trans[0][0] is paid at each boundary
+    Ct, _ = orc.dp(t, m, x, w.M)
+    ct, cm = np.cumsum(t[:, 0]), np.cumsum(m[:, 0])
+    for l in range(12):
+        expect = np.where(np.arange(201) >= cm[l], ct[l] + 777 * l, INF)
+        assert (Ct[l, :, 0] == expect).all()
+
+
+def test_zero_transition_is_multiple_choice_knapsack(orc):
+    # With trans = 0 the strategy of the previous layer does not matter:
+    # K[l][m] = min_s ( K[l-1][m-mem(l,s)] + time(l,s) ), the textbook multiple-choice knapsack.
+    w = inputs.random_tables(11, 1, 10, 6, 180, mem_lo=1, mem_hi=40)
+    t, m, x = w.time_q[0].astype(np.int64), w.mem_q[0], np.zeros((6, 6), np.int32)
+    Ct, _ = orc.dp(t, m, x, w.M)
+    K = np.full(181, 0, np.int64)
+    big = np.int64(10) ** 15
+    for l in range(10):
+        Kn = np.full(181, big)
+        for s in range(6):
+            sh = np.full(181, big)
+            sh[m[l, s]:] = K[:181 - m[l, s]] + t[l, s]
+            Kn = np.minimum(Kn, sh)
+        K = Kn
+        got = Ct[l].min(axis=1).astype(np.int64)
+        assert (np.where(K >= big, INF, K) == got).all()
+
+
+def test_zero_memory_is_layered_shortest_path(orc):
+    # With mem = 0 the budget is irrelevant and the search is a shortest path through an L x S trellis.
+    L, S = 14, 9
+    w = inputs.random_tables(21, 1, L, S, 5, mem_lo=0, mem_hi=0)
+    t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
+    assert (m == 0).all()
+    n = L * S + 1                      # node l*S+s, plus a source
+    rows, cols, vals = [], [], []
+    for s in range(S):
+        rows.append(L * S); cols.append(s); vals.append(int(t[0, s]))
+    for l in range(1, L):
+        for a in range(S):
+            for c in range(S):
+                rows.append((l - 1) * S + a); cols.append(l * S + c); vals.append(int(x[a, c]) + int(t[l, c]))
+    g = sp.csr_matrix((vals, (rows, cols)), shape=(n, n))
+    dist = dijkstra(g, directed=True, indices=L * S)
+    Ct, _ = orc.dp(t, m, x, w.M)
+    for mcol in (0, 5):
+        assert (Ct[:, mcol, :].reshape(-1) == dist[:L * S].astype(np.int64)).all()
+
+
+def test_memory_edge_cases(orc):
+    # mem > M makes a (layer, strategy) unusable at every budget; mem = 0 is legal.
+    time = np.array([[1, 2], [3, 4]]); trans = np.zeros((2, 2), int)
+    mem = np.array([[0, 50], [50, 0]])
+    Ct, At = orc.dp(time, mem, trans, 10)
+    assert (Ct[0, :, 0] == 1).all() and (Ct[0, :, 1] == INF).all()
+    assert (Ct[1, :, 0] == INF).all() and (Ct[1, :, 1] == 5).all()
+    assert orc.backtrack(time, mem, trans, Ct, None, 0)[:3:1][0] == 5
+    # L = 1
+    r = orc.search(np.array([[7, 3, 3]]), np.array([[1, 2, 2]]), np.zeros((3, 3), int), 4, budget=2)
+    assert r["opt_cost"] == 3 and r["plan"].tolist() == [1] and r["mem_used"] == 2
+
+
+def test_validation(orc):
+    ok_t = np.full((3, 2), 10); ok_m = np.ones((3, 2), int); ok_x = np.zeros((2, 2), int)
+    assert orc.validate(ok_t, ok_m, ok_x) == 0
+    bad = ok_t.copy(); bad[1, 1] = -1
+    assert orc.validate(bad, ok_m, ok_x) == orc.BAD_INPUT
+    bad = ok_m.copy(); bad[0, 0] = -5
+    assert orc.validate(ok_t, bad, ok_x) == orc.BAD_INPUT
+    bad = ok_x.copy(); bad[1, 0] = -1
+    assert orc.validate(ok_t, ok_m, bad) == orc.BAD_INPUT
+    # 3 * max_time + 2 * max_trans must stay below 2^30 - 1
+    big = np.full((3, 2), (INF - 1) // 3)
+    assert orc.validate(big, ok_m, ok_x) == 0
+    assert orc.validate(big, ok_m, np.array([[0, 1], [0, 0]])) == 0               # ...820 + 2 = 2^30 - 2
+    assert orc.validate(big, ok_m, np.array([[0, 2], [0, 0]])) == orc.OVERFLOW_RISK
+    r = orc.search(big, ok_m, np.array([[0, 2], [0, 0]]), 5)
+    assert r["status"] == orc.OVERFLOW_RISK and r["opt_cost"] == INF and (r["plan"] == -1).all()
+
+
+def test_generated_workloads_are_valid(orc):
+    w = inputs.config4(B=3)
+    assert w.time_q.shape == (3, 48, 32) and w.mem_q.min() >= 8 and w.mem_q.max() <= 128
+    assert w.trans_q.min() >= 0 and w.trans_q.max() <= 50000 and (w.trans_q[:, np.arange(32), np.arange(32)] > 0).any()
+    # log-normal(ln 5e5, 0.5): median 5e5, log-std 0.5
+    lt = np.log(inputs.config4(B=16).time_q.astype(np.float64))
+    assert abs(np.median(lt) - np.log(5e5)) < 0.02 and abs(lt.std() - 0.5) < 0.01
+    for i in range(3):
+        assert orc.validate(w.time_q[i], w.mem_q[i], w.trans_q[i]) == 0
+    # prefixes of the batch are stable
+    assert (inputs.config4(B=2).time_q == w.time_q[:2]).all()
+    w0 = inputs.config0()
+    assert (w0.trans_q[0].diagonal() == 0).all() and w0.cells == 1560 and w0.relaxations == 7020
