@@ -1,0 +1,200 @@
+/*
+ * galv.h — C boundary of the B200 strategy-search library (libgalv.so).
+ *
+ * The library runs the hot path of a hybrid-parallel strategy selector for
+ * transformer training (the "Dynamic Strategy Selector" of the paper's
+ * Section 3: profiler statistics -> performance model -> dynamic-programming
+ * search for a per-layer plan; per-layer strategies are the paper's Section 2,
+ * "Layer-Specific Parallelism Optimization"):
+ *
+ *   galv_eval_costs   cost model for every (instance, layer, strategy), fp64 -> int32
+ *   galv_dp_search    layer-wise min-plus recurrence under a memory budget
+ *   galv_backtrack    optimum at a budget and the per-layer plan
+ *
+ * for a batch of B independent search instances on one GPU (sm_100a).
+ *
+ * Conventions
+ *  - Every function returning int returns GALV_OK (0) or a negative error code.
+ *    No exceptions, no exit(), no device trap.
+ *  - Unless a parameter says "host", array pointers are DEVICE pointers owned by
+ *    the caller, 16-byte aligned.  The library allocates no device memory;
+ *    scratch comes from a caller-provided workspace sized by a query call.
+ *  - Work is enqueued on the caller's stream (a cudaStream_t passed as void*,
+ *    NULL = default stream) and is asynchronous; errors the host can detect are
+ *    returned at once, conditions found on the device land in status[B].
+ *  - A context belongs to one host thread at a time.
+ *
+ * Notation: instance i has L[i] <= Lmax layers; S strategies; budget columns
+ * m = 0..M inclusive, stored with pitch m_pitch (multiple of 32, >= M+1).
+ * Integer tables: time_q, mem_q [B][Lmax][S]; trans_q [B][S][S] with row = the
+ * previous layer's strategy s', column = this layer's strategy s.
+ * DP tables: C int32 [B][Lmax][S][m_pitch] (m fastest), A uint8 same dims.
+ */
+#ifndef GALV_H
+#define GALV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GALV_INF 1073741823 /* 2^30-1: +infinity of the cost tables, absorbing */
+
+/* return codes */
+#define GALV_OK 0
+#define GALV_ERR_INVALID_ARG (-1) /* NULL required pointer, limits violated, flags inconsistent with tables */
+#define GALV_ERR_UNSUPPORTED (-2) /* device is not compute capability 10.x */
+#define GALV_ERR_WORKSPACE (-3)   /* workspace NULL, misaligned or too small */
+#define GALV_ERR_CUDA (-4)        /* a CUDA call failed; text in galv_last_error */
+#define GALV_ERR_TIMEOUT (-5)     /* a bounded device-side wait ran out */
+
+/* per-instance status bits (status[B], device) */
+#define GALV_STATUS_INFEASIBLE 1    /* no plan fits the budget (not an error) */
+#define GALV_STATUS_BAD_INPUT 2     /* negative entry, L[i] out of 1..Lmax, bad descriptor */
+#define GALV_STATUS_OVERFLOW_RISK 4 /* a path sum could reach GALV_INF */
+#define GALV_STATUS_TIMEOUT 8       /* a bounded device-side wait ran out while this batch ran */
+
+/* shape.flags */
+#define GALV_STORE_C_FULL 1 /* keep every layer of C (needed to backtrack without A) */
+#define GALV_STORE_ARGMIN 2 /* write the argmin table A */
+#define GALV_KERNEL_REFERENCE 256 /* run the recurrence with the simple one-thread-per-cell kernel (slow; cross-checks) */
+
+typedef struct galv_ctx galv_ctx;
+
+/* limits: 1<=B, 1<=S<=256, 1<=Lmax<=65535, 0<=M<2^24, m_pitch>=M+1, m_pitch%32==0 */
+typedef struct { int32_t B, Lmax, S, M, m_pitch, flags; } galv_shape;
+
+/* One layer as the model profiler would describe it (80 bytes).
+ * FLOPs forward = c_lin*b*seq*h^2 + c_attn*b*seq^2*h; parameters = p_coef*h^2;
+ * n_ar tensor-parallel all-reduces per step; activation bytes
+ * seq*b*h*(act_rep + act_tp/tp) + act_attn*heads*seq^2*b/tp. */
+typedef struct { double h, seq, heads, c_lin, c_attn, p_coef, n_ar, act_rep, act_tp, act_attn; } galv_layer_desc;
+/* One candidate strategy (32 bytes): tensor-parallel ways, data-parallel replicas,
+ * ZeRO stage 0..3, activation checkpointing 0/1, sequence parallelism 0/1,
+ * and the divisor that turns the instance batch b into the per-replica batch. */
+typedef struct { int32_t tp, dp, zero, ckpt, sp, _pad; double batch_div; } galv_strategy_desc;
+/* One search instance (64 bytes): micro-batch, in-flight micro-batches held in
+ * memory, FLOP/s, tp and dp link bytes/s, bytes per element, bytes per memory
+ * bin, nanoseconds per integer time unit. */
+typedef struct { double b, act_mult, flops_rate, bw_tp, bw_dp, bytes_per_elem, bin_bytes, time_unit_ns; } galv_inst_params;
+
+/* Create a context on CUDA device `device_ordinal` (must be compute capability
+ * 10.x).  Allocates host memory only.  Destroy with galv_destroy. */
+int galv_create(galv_ctx** out, int device_ordinal);
+int galv_destroy(galv_ctx* ctx);
+/* Static text for a return code. */
+const char* galv_strerror(int code);
+/* Detail of the last failure on this context (valid until the next call on it). */
+const char* galv_last_error(const galv_ctx* ctx);
+
+/*
+ * Cost model (Section 3: the selector combines the model profiler's per-layer
+ * shapes/FLOPs, the hardware profiler's memory and bandwidth and the dataset
+ * profiler's batch into a performance model).  For every instance i, layer
+ * l < L[i] and strategy s, in IEEE double without fused multiply-add:
+ *   time_s    = compute/(tp*flops_rate) + tensor-parallel ring all-reduce + gradient ring all-reduce
+ *   mem_bytes = optimizer/parameter state under the ZeRO stage + act_mult * activations
+ *   time_q = rint(time_s*1e9/time_unit_ns), mem_q = ceil(mem_bytes/bin_bytes), both saturating at 2^30
+ * and for every (s', s): trans_q = rint(reshard_s*1e9/time_unit_ns), the time to
+ * re-lay-out one activation of layer 0's shape between the two tensor-parallel layouts.
+ *
+ * L [B] layers per instance; layers [B][Lmax] with layer_stride_B = Lmax, or one
+ * shared row with layer_stride_B = 0; strat [S]; inst [B].
+ * time_s, mem_bytes [B][Lmax][S] may be NULL.  Entries of layers l >= L[i] are left untouched.
+ * status[i] is set to 0, or GALV_STATUS_BAD_INPUT when L[i] is outside 1..Lmax
+ * (nothing is written for that instance).
+ */
+int galv_eval_costs(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                    const galv_layer_desc* layers, int64_t layer_stride_B,
+                    const galv_strategy_desc* strat, const galv_inst_params* inst,
+                    double* time_s, double* mem_bytes,
+                    int32_t* time_q, int32_t* mem_q, int32_t* trans_q,
+                    int32_t* status, void* stream);
+
+/* Bytes of workspace galv_dp_search needs for `shape` (0 on invalid shape). */
+size_t galv_dp_workspace_bytes(const galv_ctx* ctx, const galv_shape* shape);
+
+/*
+ * The search (Section 3: "a dynamic programming algorithm to find an optimal
+ * strategy given a performance model"), for every instance:
+ *   C[0][m][s] = time(0,s)                      if mem(0,s) <= m, else GALV_INF
+ *   C[l][m][s] = time(l,s) + min_{s'} ( C[l-1][m-mem(l,s)][s'] + trans(s',s) )
+ * GALV_INF where m < mem(l,s) or every candidate is GALV_INF.  A[l][m][s] is the
+ * lowest minimising s' (255 for GALV_INF cells and on layer 0).
+ *
+ * Before the recurrence every instance is validated: entries >= 0, L[i] in
+ * 1..Lmax, and sum_l max_s time + (L-1)*max trans < GALV_INF.  status[i] is set
+ * to 0 or to BAD_INPUT / OVERFLOW_RISK; flagged instances are skipped (their
+ * tables are left untouched) and never cause an out-of-range access.
+ *
+ * C       [B][Lmax][S][m_pitch] iff GALV_STORE_C_FULL, else NULL
+ * A       same dims, uint8, iff GALV_STORE_ARGMIN, else NULL
+ * C_last  [B][S][m_pitch], always written: layer L[i]-1 of instance i
+ * Pad columns M < m < m_pitch are written as GALV_INF / 255.
+ * workspace: 256-byte aligned, at least galv_dp_workspace_bytes(shape) bytes,
+ * overwritten by every call (calls sharing a workspace must not overlap).
+ * Enqueues one small launch per layer; nothing synchronises the host, so the
+ * call may be captured in a CUDA graph.
+ */
+int galv_dp_search(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                   const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,
+                   int32_t* C, uint8_t* A, int32_t* C_last,
+                   void* workspace, size_t workspace_bytes,
+                   int32_t* status, void* stream);
+
+/*
+ * Optimum and plan (Section 3: the selector's output is a per-layer
+ * parallelism plan).  For every instance, at budget[i] (NULL: M):
+ *   opt_cost = min_s C_last[budget][s], lowest s on ties (GALV_INF if none is finite);
+ *   plan walks back from the last layer taking, at each layer, the lowest s'
+ *   that attains the cell's minimum (read from A when given, otherwise found
+ *   again from C); mem_used = sum_l mem(l, plan[l]).
+ * Needs A, or C with GALV_STORE_C_FULL; with neither, plan must be NULL and
+ * only opt_cost is produced.  status[i]: the INFEASIBLE bit is set or cleared;
+ * instances flagged by the search get opt_cost = GALV_INF and plan = -1.
+ * plan [B][Lmax], -1 beyond L[i] and when infeasible; budget values must be in 0..M.
+ */
+int galv_backtrack(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                   const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,
+                   const int32_t* C, const uint8_t* A, const int32_t* C_last,
+                   const int32_t* budget,
+                   int32_t* opt_cost, int32_t* plan, int32_t* mem_used,
+                   int32_t* status, void* stream);
+
+/* Bytes of device arena galv_search_host needs (0 on invalid shape). */
+size_t galv_search_host_arena_bytes(const galv_ctx* ctx, const galv_shape* shape, int with_model);
+
+/*
+ * The whole path from HOST buffers: copies the inputs to the device arena, runs
+ * galv_eval_costs (when layers != NULL) or takes the host integer tables, then
+ * galv_dp_search and galv_backtrack, copies opt_cost / plan / mem_used / status
+ * back and synchronises the stream before returning.
+ * Host pointers (pinned memory makes the copies asynchronous): L, layers, strat,
+ * inst, or time_q/mem_q/trans_q; outputs opt_cost [B], plan [B][Lmax], mem_used [B],
+ * status [B].  arena: device, 256-byte aligned, galv_search_host_arena_bytes bytes.
+ * shape.flags selects the table mode as in galv_dp_search (tables live in the arena).
+ */
+int galv_search_host(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                     const galv_layer_desc* layers, int64_t layer_stride_B,
+                     const galv_strategy_desc* strat, const galv_inst_params* inst,
+                     const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,
+                     int32_t* opt_cost, int32_t* plan, int32_t* mem_used, int32_t* status,
+                     void* arena, size_t arena_bytes, void* stream);
+
+/*
+ * Integer-ALU throughput probe (the denominator of the roofline the bench
+ * reports; the paper has no counterpart).  Runs a register-only kernel of
+ * dependent-chain-free integer operations on every SM and returns operations
+ * per second in *ops_per_s (host pointer).  kind 0: fused add-then-min, counted
+ * as one operation per min-plus relaxation; kind 1: add then min written as two
+ * C statements (however the compiler lowers them), counted per relaxation;
+ * kind 2: add then xor, two plain int32 operations, both counted.  Synchronises.
+ */
+int galv_probe_int_alu(galv_ctx* ctx, int kind, int iters, double* ops_per_s, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GALV_H */

@@ -1,0 +1,146 @@
+"""ctypes binding of libgalv.so — argument marshalling only.
+
+Every step of the search runs in the library's CUDA kernels; this module turns
+torch tensors into raw device pointers and checks return codes.  PyTorch is used
+for device memory and streams, nothing else.  There is no CPU fallback: if the
+library is missing or the device is not a B200-class GPU the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+INF = 2 ** 30 - 1
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+STATUS_INFEASIBLE, STATUS_BAD_INPUT, STATUS_OVERFLOW_RISK, STATUS_TIMEOUT = 1, 2, 4, 8
+STORE_C_FULL, STORE_ARGMIN, KERNEL_REFERENCE = 1, 2, 256
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgalv.so")
+
+EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "galv_eval_costs",
+           "galv_dp_workspace_bytes", "galv_dp_search", "galv_backtrack", "galv_search_host_arena_bytes",
+           "galv_search_host", "galv_probe_int_alu")
+
+
+class galv_shape(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("B", "Lmax", "S", "M", "m_pitch", "flags")]
+
+
+class GalvError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"galv error {code}: {text}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """dlopen the in-tree library (build it first with `python -m paper_2504_03662_b200.build`)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2504_03662_b200.build`; "
+                          "there is no fallback path")
+    lib = C.CDLL(LIB_PATH)
+    vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
+    shp = C.POINTER(galv_shape)
+    lib.galv_create.argtypes = [C.POINTER(vp), C.c_int]
+    lib.galv_destroy.argtypes = [vp]
+    lib.galv_strerror.argtypes = [C.c_int]
+    lib.galv_strerror.restype = C.c_char_p
+    lib.galv_last_error.argtypes = [vp]
+    lib.galv_last_error.restype = C.c_char_p
+    lib.galv_eval_costs.argtypes = [vp, shp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.galv_dp_workspace_bytes.argtypes = [vp, shp]
+    lib.galv_dp_workspace_bytes.restype = sz
+    lib.galv_dp_search.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.galv_backtrack.argtypes = [vp, shp] + [vp] * 13
+    lib.galv_search_host_arena_bytes.argtypes = [vp, shp, C.c_int]
+    lib.galv_search_host_arena_bytes.restype = sz
+    lib.galv_search_host.argtypes = [vp, shp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.galv_probe_int_alu.argtypes = [vp, C.c_int, C.c_int, C.POINTER(C.c_double), vp]
+    _lib = lib
+    return lib
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        assert t.is_contiguous(), "tensors crossing the boundary must be contiguous"
+        return t.data_ptr()
+    return t.ctypes.data          # numpy (host buffers of galv_search_host)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def make_shape(B: int, Lmax: int, S: int, M: int, flags: int = STORE_C_FULL, m_pitch: Optional[int] = None) -> galv_shape:
+    return galv_shape(B, Lmax, S, M, (M + 1 + 31) // 32 * 32 if m_pitch is None else m_pitch, flags)
+
+
+class Galv:
+    """One library context on one CUDA device.  Methods carry the C entry points' names."""
+
+    def __init__(self, device: int = 0):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the search runs only in the CUDA library (no CPU path)")
+        self.device = device
+        h = C.c_void_p()
+        rc = self.lib.galv_create(C.byref(h), device)
+        if rc != OK:
+            raise GalvError(rc, self.lib.galv_strerror(rc).decode())
+        self.h = h
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.galv_destroy(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def _check(self, rc: int):
+        if rc != OK:
+            raise GalvError(rc, f"{self.lib.galv_strerror(rc).decode()}: {self.lib.galv_last_error(self.h).decode()}")
+
+    def galv_eval_costs(self, shape, L, layers, layer_stride_B, strat, inst, time_s, mem_bytes, time_q, mem_q,
+                        trans_q, status):
+        self._check(self.lib.galv_eval_costs(self.h, C.byref(shape), _ptr(L), _ptr(layers), layer_stride_B, _ptr(strat),
+                                             _ptr(inst), _ptr(time_s), _ptr(mem_bytes), _ptr(time_q), _ptr(mem_q),
+                                             _ptr(trans_q), _ptr(status), _stream()))
+
+    def galv_dp_workspace_bytes(self, shape) -> int:
+        return int(self.lib.galv_dp_workspace_bytes(self.h, C.byref(shape)))
+
+    def galv_dp_search(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, workspace, status):
+        self._check(self.lib.galv_dp_search(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),
+                                            _ptr(Ct), _ptr(At), _ptr(C_last), _ptr(workspace),
+                                            0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                            _ptr(status), _stream()))
+
+    def galv_backtrack(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, budget, opt_cost, plan, mem_used, status):
+        self._check(self.lib.galv_backtrack(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),
+                                            _ptr(Ct), _ptr(At), _ptr(C_last), _ptr(budget), _ptr(opt_cost), _ptr(plan),
+                                            _ptr(mem_used), _ptr(status), _stream()))
+
+    def galv_search_host_arena_bytes(self, shape, with_model: bool) -> int:
+        return int(self.lib.galv_search_host_arena_bytes(self.h, C.byref(shape), int(with_model)))
+
+    def galv_search_host(self, shape, L, layers, layer_stride_B, strat, inst, time_q, mem_q, trans_q,
+                         opt_cost, plan, mem_used, status, arena):
+        self._check(self.lib.galv_search_host(self.h, C.byref(shape), _ptr(L), _ptr(layers), layer_stride_B, _ptr(strat),
+                                              _ptr(inst), _ptr(time_q), _ptr(mem_q), _ptr(trans_q), _ptr(opt_cost),
+                                              _ptr(plan), _ptr(mem_used), _ptr(status), _ptr(arena),
+                                              arena.numel() * arena.element_size(), _stream()))
+
+    def galv_probe_int_alu(self, kind: int, iters: int = 4096) -> float:
+        out = C.c_double()
+        self._check(self.lib.galv_probe_int_alu(self.h, kind, iters, C.byref(out), _stream()))
+        return out.value

@@ -1,0 +1,522 @@
+// Layer-wise min-plus recurrence of the strategy search on sm_100a.
+//
+//   C[l][m][s] = time(l,s) + min_{s'} ( C[l-1][m-mem(l,s)][s'] + trans(s',s) )
+//
+// (Section 3 of the paper: dynamic-programming search over a performance model.)
+//
+// Per layer the work is a min-plus product G[s][m'] = min_{s'} (Cprev[s'][m'] + T[s'][s])
+// that does not depend on mem; mem only shifts where column m' is stored:
+// C[l][s][m'+mem(l,s)] = time(l,s) + G[s][m'].  So the kernel tiles like a
+// CUDA-core GEMM: an item is (instance, tile of m', block of s); warps own a
+// register tile of (TM x 32 columns) x (8 strategies); the previous layer's rows
+// are staged in shared memory by bulk async copies (TMA unit) and the S x S
+// transition rows by cp.async, double buffered over chunks of s'.  One fused
+// add-min instruction per relaxation; no tensor cores (min-plus is not a
+// multiply-add contraction).
+//
+// One launch per layer (a layer needs all of the previous one); launches are
+// plain stream work, so a caller may capture the whole search in a CUDA graph.
+
+#include "galv_internal.h"
+
+namespace {
+
+constexpr int kInf = GALV_INF;
+constexpr int TS = 8;                 // strategies per warp register tile
+constexpr int kSpinLimit = 1 << 22;   // bounded mbarrier polling (each poll may block for a while in hardware)
+
+// ---------------------------------------------------------------- PTX helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (int i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// 1-D bulk async copy global -> shared, completion counted in bytes on an mbarrier.
+// dst, src 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// ---------------------------------------------------------------- validation / schedule
+
+// One CTA per instance: entries >= 0, L in range, worst-case path sum below kInf.
+__global__ void validate_kernel(int B, int Lmax, int S, const int32_t* __restrict__ L,
+                                const int32_t* __restrict__ time_q, const int32_t* __restrict__ mem_q,
+                                const int32_t* __restrict__ trans_q, int32_t* __restrict__ status)
+{
+    const int i = blockIdx.x;
+    __shared__ long long s_sum;
+    __shared__ int s_tmax, s_bad;
+    if (threadIdx.x == 0) { s_sum = 0; s_tmax = 0; s_bad = 0; }
+    __syncthreads();
+    const int Li = L[i];
+    if (Li < 1 || Li > Lmax) {
+        if (threadIdx.x == 0) status[i] = GALV_STATUS_BAD_INPUT;
+        return;
+    }
+    long long sum = 0;
+    int bad = 0, tmax = 0;
+    const int32_t* t = time_q + (size_t)i * Lmax * S;
+    const int32_t* mq = mem_q + (size_t)i * Lmax * S;
+    for (int l = threadIdx.x; l < Li; l += blockDim.x) {
+        int mx = 0;
+        for (int s = 0; s < S; ++s) {
+            const int tv = t[l * S + s], mv = mq[l * S + s];
+            bad |= (tv < 0) | (mv < 0);
+            mx = max(mx, tv);
+        }
+        sum += mx;
+    }
+    const int32_t* x = trans_q + (size_t)i * S * S;
+    for (int k = threadIdx.x; k < S * S; k += blockDim.x) {
+        const int v = x[k];
+        bad |= (v < 0);
+        tmax = max(tmax, v);
+    }
+    atomicAdd(reinterpret_cast<unsigned long long*>(&s_sum), static_cast<unsigned long long>(sum));
+    atomicMax(&s_tmax, tmax);
+    if (bad) atomicOr(&s_bad, 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int st = 0;
+        if (s_bad) st = GALV_STATUS_BAD_INPUT;
+        else if (s_sum + (long long)(Li - 1) * s_tmax >= (long long)kInf) st = GALV_STATUS_OVERFLOW_RISK;
+        status[i] = st;
+    }
+}
+
+// Single CTA: nactive[l] = valid instances with L > l; order = valid instances, longest first.
+// scratch = hist[Lmax+2] | fill[Lmax+2], zeroed by the host before the launch.
+__global__ void schedule_kernel(int B, int Lmax, const int32_t* __restrict__ L, const int32_t* __restrict__ status,
+                                int32_t* __restrict__ order, int32_t* __restrict__ nactive, int32_t* __restrict__ scratch)
+{
+    int32_t* hist = scratch;
+    int32_t* fill = scratch + Lmax + 2;
+    for (int i = threadIdx.x; i < B; i += blockDim.x)
+        if (status[i] == 0) atomicAdd(&hist[L[i]], 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;                                   // instances with L > l, from the top down
+        for (int l = Lmax; l >= 0; --l) { nactive[l] = run; run += hist[l]; }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < B; i += blockDim.x)
+        if (status[i] == 0) {
+            const int Li = L[i];
+            order[nactive[Li] + atomicAdd(&fill[Li], 1)] = i;   // instances longer than Li come first
+        }
+}
+
+// ---------------------------------------------------------------- base layer
+
+// C[0][s][m] = time(0,s) if mem(0,s) <= m else INF; pad columns INF; A = 255.
+__global__ void base_layer_kernel(DpArgs a)
+{
+    const int i = blockIdx.z, s = blockIdx.y;
+    if (a.status[i] != 0) return;
+    const int tt = a.time_q[(size_t)i * a.Lmax * a.S + s];
+    const int mm = a.mem_q[(size_t)i * a.Lmax * a.S + s];
+    const size_t row = ((size_t)i * a.S + s) * a.m_pitch;
+    int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax * a.S + s) * a.m_pitch : a.roll + row;
+    int32_t* last = (a.L[i] == 1) ? a.C_last + row : nullptr;
+    uint8_t* ao = a.A ? a.A + ((size_t)i * a.Lmax * a.S + s) * a.m_pitch : nullptr;
+    for (int m = blockIdx.x * blockDim.x + threadIdx.x; m < a.m_pitch; m += gridDim.x * blockDim.x) {
+        const int v = (m <= a.M && mm <= m) ? tt : kInf;
+        out[m] = v;
+        if (last) last[m] = v;
+        if (ao) ao[m] = 255;
+    }
+}
+
+// ---------------------------------------------------------------- reference layer kernel (one thread per cell)
+
+__global__ void layer_reference_kernel(DpArgs a, int l)
+{
+    const int mchunks = (a.m_pitch + blockDim.x - 1) / blockDim.x;
+    const int oi = blockIdx.x / mchunks;
+    if (oi >= a.nactive[l]) return;
+    const int i = a.order[oi], s = blockIdx.y;
+    const int m = (blockIdx.x % mchunks) * blockDim.x + threadIdx.x;
+    if (m >= a.m_pitch) return;
+    const size_t slice = (size_t)a.S * a.m_pitch;
+    const int32_t* prev = a.C ? a.C + ((size_t)i * a.Lmax + (l - 1)) * slice : a.roll + ((size_t)((l - 1) & 1) * a.B + i) * slice;
+    int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
+    const int32_t* T = a.trans_q + (size_t)i * a.S * a.S;
+    const int mm = a.mem_q[((size_t)i * a.Lmax + l) * a.S + s];
+    const int tt = a.time_q[((size_t)i * a.Lmax + l) * a.S + s];
+    int best = kInf, arg = 255;
+    if (m <= a.M && mm <= m) {
+        const int mp = m - mm;
+        for (int sp = 0; sp < a.S; ++sp) {
+            const int c = prev[(size_t)sp * a.m_pitch + mp];
+            if (c < kInf) {
+                const int v = c + T[sp * a.S + s];
+                if (v < best) { best = v; arg = sp; }
+            }
+        }
+    }
+    const int v = best < kInf ? best + tt : kInf;
+    out[(size_t)s * a.m_pitch + m] = v;
+    if (a.L[i] == l + 1) a.C_last[((size_t)i * a.S + s) * a.m_pitch + m] = v;
+    if (a.A) a.A[(((size_t)i * a.Lmax + l) * a.S + s) * a.m_pitch + m] = (uint8_t)arg;
+}
+
+// ---------------------------------------------------------------- tiled layer kernel
+
+struct Item { int i, mt, sb; };
+
+__device__ __forceinline__ Item decode_item(long long item, const DpPlan& pl, const int32_t* __restrict__ order) {
+    const int per = pl.ntiles_m * pl.nsb;
+    const int oi = (int)(item / per);
+    const int r = (int)(item - (long long)oi * per);
+    Item it;
+    it.i = order[oi];
+    it.mt = r / pl.nsb;
+    it.sb = r - it.mt * pl.nsb;
+    return it;
+}
+
+template <int TM, bool ARG>
+__global__ void __launch_bounds__(512, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[2];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nthreads = blockDim.x;
+    const int S = a.S, M = a.M, m_pitch = a.m_pitch;
+    const int TMB = pl.tmb, SB = pl.sb, KS = pl.ks, NKC = pl.nkc;
+    const int sg = warp % pl.nsg, ms = warp / pl.nsg;
+
+    const long long nitems = (long long)a.nactive[l] * pl.ntiles_m * pl.nsb;
+    if ((long long)blockIdx.x >= nitems) return;
+
+    int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
+    const int stage_elems = KS * (TMB + SB);
+
+    if (tid == 0) {
+        mbar_init(&full_bar[0], 1);
+        mbar_init(&full_bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const size_t slice = (size_t)S * m_pitch;
+    const bool vec16 = (S & 3) == 0;
+
+    // Stage one chunk (item, kc): rows k0..k0+kn of the previous layer's slice, columns
+    // [m0, m0+w), by bulk copies from warp 0; the matching rows of trans by cp.async from all.
+    auto issue_load = [&](long long item, int kc, int st) {
+        const Item it = decode_item(item, pl, a.order);
+        const int m0 = it.mt * TMB;
+        const int w = min(TMB, m_pitch - m0);
+        const int k0 = kc * KS;
+        const int kn = min(KS, S - k0);
+        const int sb0 = it.sb * SB;
+        int32_t* cs = stage0 + st * stage_elems;
+        int32_t* ts = cs + KS * TMB;
+        const int32_t* prev = (a.C ? a.C + ((size_t)it.i * a.Lmax + (l - 1)) * slice
+                                   : a.roll + ((size_t)((l - 1) & 1) * a.B + it.i) * slice)
+                              + (size_t)k0 * m_pitch + m0;
+        if (warp == 0) {
+            if (lane == 0) mbar_expect_tx(&full_bar[st], (uint32_t)kn * w * 4u);
+            __syncwarp();
+            for (int r = lane; r < kn; r += 32)
+                bulk_g2s(cs + r * TMB, prev + (size_t)r * m_pitch, (uint32_t)w * 4u, &full_bar[st]);
+        }
+        const int32_t* T = a.trans_q + (size_t)it.i * S * S + (size_t)k0 * S + sb0;
+        if (vec16) {
+            const int q = SB >> 2;
+            for (int e = tid; e < kn * q; e += nthreads) {
+                const int r = e / q, c = (e - r * q) << 2;
+                if (sb0 + c < S) cp_async16(ts + r * SB + c, T + (size_t)r * S + c);
+            }
+        } else {
+            for (int e = tid; e < kn * SB; e += nthreads) {
+                const int r = e / SB, c = e - r * SB;
+                if (sb0 + c < S) cp_async4(ts + r * SB + c, T + (size_t)r * S + c);
+            }
+        }
+        cp_async_commit();
+    };
+
+    long long ld_item = blockIdx.x; int ld_kc = 0;       // load cursor
+    long long cp_item = blockIdx.x; int cp_kc = 0;       // compute cursor
+    issue_load(ld_item, ld_kc, 0);
+    if (++ld_kc == NKC) { ld_kc = 0; ld_item += gridDim.x; }
+
+    int acc[TM][TS];
+    int arg[ARG ? TM : 1][ARG ? TS : 1];
+    (void)arg;
+
+    for (int iter = 0; cp_item < nitems; ++iter) {
+        const int st = iter & 1;
+        cp_async_wait_all();
+        if (!mbar_wait(&full_bar[st], (iter >> 1) & 1)) {
+            // Give up cleanly: flag the error; a second bounded wait lets copies in flight land.
+            if (tid == 0) atomicExch(a.err, 1);
+            mbar_wait(&full_bar[st], (iter >> 1) & 1);
+            return;
+        }
+        __syncthreads();      // trans rows visible to all; everyone is done with the other stage
+        if (ld_item < nitems) {
+            issue_load(ld_item, ld_kc, st ^ 1);
+            if (++ld_kc == NKC) { ld_kc = 0; ld_item += gridDim.x; }
+        }
+
+        const Item it = decode_item(cp_item, pl, a.order);
+        const int m0 = it.mt * TMB;
+        const int k0 = cp_kc * KS;
+        const int kn = min(KS, S - k0);
+        const int mw = m0 + ms * (32 * TM);                 // first column of this warp
+        // 32-column groups of this warp that hold at least one column <= M
+        const int nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
+
+        if (cp_kc == 0) {
+#pragma unroll
+            for (int j = 0; j < TM; ++j)
+#pragma unroll
+                for (int u = 0; u < TS; ++u) {
+                    acc[j][u] = 0x7fffffff;
+                    if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = 255;
+                }
+        }
+
+        const int32_t* cs = stage0 + st * stage_elems + ms * (32 * TM) + lane;
+        const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
+
+        if (nj == TM) {
+#pragma unroll 2
+            for (int k = 0; k < kn; ++k) {
+                int c[TM];
+#pragma unroll
+                for (int j = 0; j < TM; ++j) c[j] = cs[k * TMB + j * 32];
+                const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
+                const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
+                const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                for (int j = 0; j < TM; ++j)
+#pragma unroll
+                    for (int u = 0; u < TS; ++u) {
+                        if (ARG) {
+                            const int cand = c[j] + t[u];
+                            if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
+                        } else {
+                            acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                        }
+                    }
+            }
+        } else if (nj > 0) {
+            // ragged last tile: only the first nj column groups carry work
+            for (int k = 0; k < kn; ++k) {
+                const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
+                const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
+                const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                for (int j = 0; j < TM; ++j)
+                    if (j < nj) {
+                        const int c = cs[k * TMB + j * 32];
+#pragma unroll
+                        for (int u = 0; u < TS; ++u) {
+                            const int cand = c + t[u];
+                            if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
+                        }
+                    }
+            }
+        }
+
+        if (cp_kc == NKC - 1) {
+            // Epilogue: column m' of strategy s lands at m = m' + mem(l,s).
+            const int i = it.i;
+            const bool is_last = (a.L[i] == l + 1);
+            int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
+            int32_t* last = a.C_last + (size_t)i * slice;
+            uint8_t* aout = ARG ? a.A + ((size_t)i * a.Lmax + l) * slice : nullptr;
+            const size_t qrow = ((size_t)i * a.Lmax + l) * S;
+            const int sb0 = it.sb * SB;
+#pragma unroll
+            for (int u = 0; u < TS; ++u) {
+                const int s = sb0 + sg * TS + u;
+                if (s < S) {
+                    const int mm = __ldg(a.mem_q + qrow + s);
+                    const int tt = __ldg(a.time_q + qrow + s);
+#pragma unroll
+                    for (int j = 0; j < TM; ++j) {
+                        const int mp = mw + j * 32 + lane;
+                        if (j < nj && mp <= M && mm <= M - mp) {
+                            const size_t o = (size_t)s * m_pitch + (mp + mm);
+                            const int g = acc[j][u];
+                            const int v = g >= kInf ? kInf : g + tt;
+                            out[o] = v;
+                            if (is_last) last[o] = v;
+                            if (ARG) aout[o] = (uint8_t)(g >= kInf ? 255 : arg[ARG ? j : 0][ARG ? u : 0]);
+                        }
+                    }
+                }
+            }
+            if (it.mt == 0) {
+                // Cells no column maps to: m < mem(l,s), and the pad columns.
+                const int nw = nthreads >> 5;
+                for (int s = sb0 + warp; s < min(S, sb0 + SB); s += nw) {
+                    const int mm = __ldg(a.mem_q + qrow + s);
+                    const int lo = min(mm, M + 1);
+                    const size_t o = (size_t)s * m_pitch;
+                    for (int m = lane; m < m_pitch; m += 32)
+                        if (m < lo || m > M) {
+                            out[o + m] = kInf;
+                            if (is_last) last[o + m] = kInf;
+                            if (ARG) aout[o + m] = 255;
+                        }
+                }
+            }
+            cp_kc = 0;
+            cp_item += gridDim.x;
+        } else {
+            ++cp_kc;
+        }
+    }
+}
+
+// Sets the TIMEOUT bit everywhere when a bounded wait ran out.
+__global__ void finalize_kernel(int B, const int32_t* err, int32_t* status)
+{
+    if (*err == 0) return;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < B; i += gridDim.x * blockDim.x)
+        status[i] |= GALV_STATUS_TIMEOUT;
+}
+
+template <int TM, bool ARG>
+cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st)
+{
+    layer_tiled_kernel<TM, ARG><<<pl.grid, pl.threads, pl.smem, st>>>(a, pl, l);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------- host side
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+WsLayout galv_ws_layout(const galv_shape* sh)
+{
+    WsLayout w;
+    size_t off = 0;
+    w.order = off;   off = align256(off + (size_t)sh->B * 4);
+    w.nactive = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
+    w.scratch = off; off = align256(off + (size_t)2 * (sh->Lmax + 2) * 4);
+    w.err = off;     off = align256(off + 4);
+    w.roll = off;
+    if (!(sh->flags & GALV_STORE_C_FULL)) off = align256(off + (size_t)2 * sh->B * sh->S * sh->m_pitch * 4);
+    w.total = off;
+    return w;
+}
+
+bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
+{
+    const int S = sh->S;
+    const int spad = (S + TS - 1) / TS * TS;
+    pl->tm = 4;
+    pl->nsb = (spad + 63) / 64;
+    pl->sb = ((S + pl->nsb - 1) / pl->nsb + TS - 1) / TS * TS;
+    pl->nsg = pl->sb / TS;
+    pl->nms = 16 / pl->nsg;
+    if (pl->nms < 1) pl->nms = 1;
+    pl->tmb = pl->nms * 32 * pl->tm;
+    pl->threads = pl->nsg * pl->nms * 32;
+    // two stages of ks * (tmb + sb) ints must fit the opt-in shared memory
+    const int budget = (ctx->smem_optin - 1024) / 2;
+    int ks = budget / ((pl->tmb + pl->sb) * 4);
+    if (ks > S) ks = S;
+    if (ks > 64) ks = 64;
+    if (ks < 1) return false;
+    pl->ks = ks;
+    pl->nkc = (S + ks - 1) / ks;
+    pl->ntiles_m = (sh->M + 1 + pl->tmb - 1) / pl->tmb;
+    pl->smem = 2 * ks * (pl->tmb + pl->sb) * 4;
+    const long long items = (long long)sh->B * pl->ntiles_m * pl->nsb;
+    pl->grid = (int)(items < ctx->num_sms ? items : ctx->num_sms);
+    return true;
+}
+
+cudaError_t galv_dp_configure(const galv_ctx* ctx)
+{
+    cudaError_t e;
+    e = cudaFuncSetAttribute(layer_tiled_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(layer_tiled_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 1024);
+    return e;
+}
+
+cudaError_t galv_dp_launch(const galv_ctx* ctx, const galv_shape* sh, const DpArgs& a, cudaStream_t st)
+{
+    cudaError_t e;
+    const int B = a.B, Lmax = a.Lmax, S = a.S;
+    e = cudaMemsetAsync(a.scratch, 0, (size_t)2 * (Lmax + 2) * 4, st);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(a.err, 0, 4, st);
+    if (e != cudaSuccess) return e;
+    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.L, a.time_q, a.mem_q, a.trans_q, a.status);
+    schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.L, a.status, a.order, a.nactive, a.scratch);
+    {
+        int gx = (a.m_pitch + 255) / 256;
+        if (gx > 8) gx = 8;
+        for (int b0 = 0; b0 < B; b0 += 65535) {           // grid.z limit
+            DpArgs s = a;
+            const int nb = (B - b0 < 65535) ? B - b0 : 65535;
+            s.L += b0; s.status += b0;
+            s.time_q += (size_t)b0 * Lmax * S; s.mem_q += (size_t)b0 * Lmax * S;
+            if (s.C) s.C += (size_t)b0 * Lmax * S * a.m_pitch;
+            if (s.A) s.A += (size_t)b0 * Lmax * S * a.m_pitch;
+            s.C_last += (size_t)b0 * S * a.m_pitch;
+            s.roll += (size_t)b0 * S * a.m_pitch;
+            base_layer_kernel<<<dim3(gx, S, nb), 256, 0, st>>>(s);
+        }
+    }
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+
+    const bool reference = (sh->flags & GALV_KERNEL_REFERENCE) != 0;
+    DpPlan pl;
+    if (!reference && !galv_dp_make_plan(ctx, sh, &pl)) return cudaErrorInvalidConfiguration;
+    for (int l = 1; l < Lmax; ++l) {
+        if (reference) {
+            const int mchunks = (a.m_pitch + 255) / 256;
+            layer_reference_kernel<<<dim3((unsigned)((size_t)B * mchunks), S, 1), 256, 0, st>>>(a, l);
+            e = cudaGetLastError();
+        } else {
+            e = a.A ? launch_tiled<4, true>(a, pl, l, st) : launch_tiled<4, false>(a, pl, l, st);
+        }
+        if (e != cudaSuccess) return e;
+    }
+    finalize_kernel<<<(B + 255) / 256, 256, 0, st>>>(B, a.err, a.status);
+    return cudaGetLastError();
+}

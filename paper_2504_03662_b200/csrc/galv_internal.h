@@ -1,0 +1,68 @@
+// Internal declarations shared by the translation units of libgalv.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "galv.h"
+
+struct galv_ctx {
+    int device;
+    int num_sms;
+    int smem_optin;      // max dynamic shared memory per block (bytes)
+    char err[512];
+};
+
+// How one layer of the recurrence is cut into work items (host-chosen, passed to the kernels).
+struct DpPlan {
+    int tm;        // 32-column groups per warp (register tile height)
+    int sb;        // strategies per item (s-block), multiple of 8
+    int nsb;       // s-blocks
+    int nsg;       // warps along s  (= sb / 8)
+    int nms;       // warps along m
+    int tmb;       // budget columns per item = nms * 32 * tm
+    int ks;        // previous-layer strategies staged per pipeline stage
+    int nkc;       // stages per item = ceil(S / ks)
+    int ntiles_m;  // ceil((M+1) / tmb)
+    int threads;   // nsg * nms * 32
+    int smem;      // dynamic shared memory bytes
+    int grid;      // resident CTAs
+};
+
+struct DpArgs {
+    int B, Lmax, S, M, m_pitch;
+    const int32_t* L;
+    const int32_t* time_q;
+    const int32_t* mem_q;
+    const int32_t* trans_q;
+    int32_t* C;          // full table or NULL
+    uint8_t* A;          // argmin table or NULL
+    int32_t* C_last;
+    int32_t* roll;       // [2][B][S][m_pitch] when C == NULL
+    int32_t* order;      // [B]   valid instances, longest first
+    int32_t* nactive;    // [Lmax+1] instances with L > l
+    int32_t* scratch;    // [2*(Lmax+2)] histogram / fill counters
+    int32_t* err;        // device error flag
+    int32_t* status;
+};
+
+// workspace carve-up (offsets in bytes, all 256-aligned)
+struct WsLayout { size_t order, nactive, scratch, err, roll, total; };
+WsLayout galv_ws_layout(const galv_shape* sh);
+
+bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* plan);
+cudaError_t galv_dp_configure(const galv_ctx* ctx);
+cudaError_t galv_dp_launch(const galv_ctx* ctx, const galv_shape* sh, const DpArgs& a, cudaStream_t st);
+cudaError_t galv_backtrack_launch(const galv_shape* sh, const int32_t* L, const int32_t* time_q,
+                                  const int32_t* mem_q, const int32_t* trans_q, const int32_t* C,
+                                  const uint8_t* A, const int32_t* C_last, const int32_t* budget,
+                                  int32_t* opt_cost, int32_t* plan, int32_t* mem_used, int32_t* status,
+                                  cudaStream_t st);
+cudaError_t galv_costs_launch(const galv_shape* sh, const int32_t* L, const galv_layer_desc* layers,
+                              int64_t layer_stride_B, const galv_strategy_desc* strat,
+                              const galv_inst_params* inst, double* time_s, double* mem_bytes,
+                              int32_t* time_q, int32_t* mem_q, int32_t* trans_q, int32_t* status,
+                              cudaStream_t st);
+cudaError_t galv_probe_launch(const galv_ctx* ctx, int kind, int iters, int32_t* sink, cudaStream_t st,
+                              long long* ops);

@@ -1,0 +1,291 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, through the C boundary."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+
+from paper_2504_03662_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+INF = 2 ** 30 - 1
+
+
+@pytest.fixture(scope="module")
+def galv():
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    g = gb.Galv(0)
+    yield g
+    g.close()
+
+
+def oracle_tables(orc, w):
+    """Integer tables of every instance from the oracle's own cost model (or the workload's)."""
+    if not w.has_model:
+        return w.time_q, w.mem_q, w.trans_q
+    tq = np.zeros((w.B, w.Lmax, w.S), np.int32); mq = np.zeros_like(tq); xq = np.zeros((w.B, w.S, w.S), np.int32)
+    for i in range(w.B):
+        Li = int(w.L[i])
+        _, _, t, m, x = orc.eval_costs(w.layers[0 if w.layers.shape[0] == 1 else i], w.strat, w.inst[i], Li)
+        tq[i, :Li], mq[i, :Li], xq[i] = t, m, x
+    return tq, mq, xq
+
+
+def oracle_search_many(orc, w, tq, mq, xq, idx, use_A=False):
+    def one(i):
+        Li = int(w.L[i])
+        return orc.search(tq[i, :Li], mq[i, :Li], xq[i], w.M, use_A=use_A)
+    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+        return dict(zip(idx, ex.map(one, idx)))
+
+
+def check_batch(orc, galv, w, flags, idx=None, tables=True, budget=None):
+    """Run the GPU path on the whole batch and compare instances `idx` with the oracle."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    sb = SearchBuffers(galv, w, flags)
+    tq, mq, xq = oracle_tables(orc, w)
+    if w.has_model:
+        sb.eval_costs()
+        torch.cuda.synchronize()
+        for name, ref, got in (("time_q", tq, sb.time_q), ("mem_q", mq, sb.mem_q), ("trans_q", xq, sb.trans_q)):
+            g = got.cpu().numpy()
+            for i in range(w.B):
+                Li = int(w.L[i]) if name != "trans_q" else w.S
+                assert (g[i, :Li] == ref[i, :Li]).all(), (name, i)
+    sb.dp_search()
+    bud = None if budget is None else torch.from_numpy(np.asarray(budget, np.int32)).to(sb.dev)
+    sb.backtrack(bud)
+    res = sb.results()
+    idx = list(range(w.B)) if idx is None else list(idx)
+    ref = oracle_search_many(orc, w, tq, mq, xq, idx)
+    for i in idx:
+        r, Li = ref[i], int(w.L[i])
+        b = w.M if budget is None else int(budget[i])
+        if budget is not None and r["C"] is not None:
+            o, p, u, st = orc.backtrack(tq[i, :Li], mq[i, :Li], xq[i], r["C"], None, b)
+            r = dict(r, opt_cost=o, plan=p, mem_used=u, status=st)
+        assert res["status"][i] == r["status"], (i, res["status"][i], r["status"])
+        assert res["opt_cost"][i] == r["opt_cost"], i
+        assert (res["plan"][i, :Li] == r["plan"]).all(), (i, res["plan"][i, :Li], r["plan"])
+        assert (res["plan"][i, Li:] == -1).all()
+        assert res["mem_used"][i] == r["mem_used"]
+        if r["C"] is None:
+            continue
+        last = sb.C_last[i, :, :w.M + 1].t().cpu().numpy()
+        assert (last == r["C"][Li - 1]).all(), i
+        assert (sb.C_last[i, :, w.M + 1:] == INF).all()
+        if tables and flags & gb.STORE_C_FULL:
+            got = sb.table(i)[:Li]
+            assert (got == r["C"]).all(), (i, np.argwhere(got != r["C"])[:5])
+        if tables and flags & gb.STORE_ARGMIN:
+            got = sb.argmin_table(i)[:Li]
+            assert (got == r["A"]).all(), (i, np.argwhere(got != r["A"])[:5])
+    return sb, res
+
+
+MODES = [1, 3, 2, 1 | 256, 3 | 256]      # full C; full C + A; rolling + A; the same with the reference kernel
+
+
+@pytest.mark.parametrize("flags", MODES)
+def test_config0_every_budget(orc, galv, flags):
+    w = inputs.config0()
+    check_batch(orc, galv, w, flags)
+    rows = [l.split() for l in open(os.path.join(os.path.dirname(__file__), "golden", "config0_bruteforce.txt"))
+            if not l.startswith("#")]
+    # all 65 budgets in one batch of 65 copies of the instance
+    w65 = inputs.Workload("config0x65", 65, w.Lmax, w.S, w.M, np.full(65, 4, np.int32),
+                          np.repeat(w.time_q, 65, 0), np.repeat(w.mem_q, 65, 0), np.repeat(w.trans_q, 65, 0))
+    sb, res = check_batch(orc, galv, w65, flags, budget=np.arange(65))
+    for r in rows:
+        b = int(r[0])
+        assert res["opt_cost"][b] == int(r[1]) and res["plan"][b].tolist() == [int(v) for v in r[4:]]
+
+
+SHAPES = [  # B, Lmax, S, M, kwargs
+    (3, 5, 1, 40, {}),
+    (4, 7, 5, 97, dict(ragged=True)),
+    (2, 6, 8, 255, {}),
+    (3, 9, 13, 300, dict(ragged=True, mem_lo=0, mem_hi=0)),            # memory-free: layered shortest path
+    (2, 4, 33, 1000, dict(dup_cols=True, time_hi=5, trans_hi=2)),      # tie-heavy, S just above a warp
+    (2, 3, 70, 513, dict(mem_hi=700)),                                 # two s-blocks; many mem > M
+    (5, 1, 6, 64, {}),                                                 # single layer
+    (2, 5, 24, 2881, dict(mem_lo=3000, mem_hi=4000)),                  # nothing fits
+    (2, 12, 32, 2048, dict(mem_lo=8, mem_hi=128, trans_hi=50000)),     # tile edge: M+1 = 4*512+1
+    (1, 3, 130, 200, {}),                                              # three s-blocks
+    (1, 3, 256, 100, dict(time_hi=100000)),                            # the largest S
+]
+
+
+@pytest.mark.parametrize("flags", [1, 3, 2])
+@pytest.mark.parametrize("k", range(len(SHAPES)))
+def test_random_shapes(orc, galv, flags, k):
+    B, Lmax, S, M, kw = SHAPES[k]
+    w = inputs.random_tables(700 + k, B, Lmax, S, M, **kw)
+    sb, res = check_batch(orc, galv, w, flags)
+    if k == 7:
+        assert (res["status"] == 1).all() and (res["opt_cost"] == INF).all()
+
+
+def test_budget_queries(orc, galv):
+    w = inputs.random_tables(31, 6, 8, 12, 400, mem_lo=1, mem_hi=90)
+    check_batch(orc, galv, w, 3, budget=[0, 50, 123, 399, 400, 200])
+
+
+def test_flagged_instances_are_skipped(orc, galv):
+    import torch
+    w = inputs.random_tables(5, 6, 4, 6, 50, ragged=True)
+    w.time_q[1, 0, 2] = -7                       # negative entry
+    w.L[2] = 0                                   # L out of range
+    w.time_q[3] = (INF - 1) // 2                 # sum could reach INF
+    w.L[3] = 4
+    w.mem_q[4, 1, :] = -1
+    w.L[4] = 4
+    w.L[5] = 9                                   # above Lmax
+    sb, res = check_batch(orc, galv, w, 3, idx=[0])
+    assert res["status"].tolist()[1:] == [2, 2, 4, 2, 2]
+    assert (res["opt_cost"][1:] == INF).all() and (res["plan"][1:] == -1).all() and (res["mem_used"][1:] == 0).all()
+    # an out-of-range budget is reported, not followed
+    sb.backtrack(torch.tensor([51, -1, 0, 0, 0, 0], dtype=torch.int32, device=sb.dev))
+    r2 = sb.results()
+    assert r2["status"][0] == 2 and r2["opt_cost"][0] == INF
+
+
+def test_config1_full(orc, galv):
+    sb, res = check_batch(orc, galv, inputs.config1(), 3)
+    assert (res["status"] == 0).all()
+
+
+def test_config2_full_ragged(orc, galv):
+    w = inputs.config2()
+    sb, res = check_batch(orc, galv, w, 1)
+    assert set(res["status"].tolist()) <= {0, 1}
+    sb, res = check_batch(orc, galv, w, 2, idx=range(0, 64, 5), tables=False)
+
+
+def test_config2_full_product_extra(orc, galv):
+    check_batch(orc, galv, inputs.config2(full_product=True), 1, idx=[3, 17, 40, 63])
+
+
+def _properties_all(orc, w, tq, mq, xq, sb, res):
+    """What holds at any size: plan cost equals the optimum, memory within budget, C_last monotone."""
+    last = sb.C_last[:, :, :w.M + 1]
+    assert bool((last[:, :, :-1] >= last[:, :, 1:]).all())
+    for i in range(w.B):
+        Li = int(w.L[i])
+        if res["status"][i] == 0:
+            c, u = orc.plan_cost(tq[i, :Li], mq[i, :Li], xq[i], res["plan"][i, :Li])
+            assert c == res["opt_cost"][i] and u == res["mem_used"][i] <= w.M
+
+
+def test_config4_full_size(orc, galv):
+    w = inputs.config4()
+    idx = [0, 1, 511, 777, 1023] + list(range(64, 1024, 64))
+    sb, res = check_batch(orc, galv, w, 1, idx=idx)
+    assert (res["status"] == 0).all()
+    _properties_all(orc, w, w.time_q, w.mem_q, w.trans_q, sb, res)
+    del sb
+    sb, res2 = check_batch(orc, galv, w, 2, idx=idx[:6], tables=False)
+    assert (res2["opt_cost"] == res["opt_cost"]).all() and (res2["plan"] == res["plan"]).all()
+
+
+def test_config3_full_size(orc, galv):
+    import torch
+    w = inputs.config3()
+    idx = [0, 37, 127]
+    sb, res = check_batch(orc, galv, w, 1, idx=idx)
+    assert (res["status"] == 0).all()
+    tq, mq, xq = oracle_tables(orc, w)
+    _properties_all(orc, w, tq, mq, xq, sb, res)
+    del sb
+    torch.cuda.empty_cache()
+
+
+def test_cost_model_fp64(orc, galv):
+    import torch
+    from paper_2504_03662_b200.search import SearchBuffers
+    for w in (inputs.config1(), inputs.config2(), inputs.config3(B=8)):
+        sb = SearchBuffers(galv, w, 1)
+        sb.eval_costs(want_fp64=True)
+        torch.cuda.synchronize()
+        ts, mb = sb.time_s.cpu().numpy(), sb.mem_bytes.cpu().numpy()
+        for i in range(w.B):
+            Li = int(w.L[i])
+            rts, rmb, *_ = orc.eval_costs(w.layers[0], w.strat, w.inst[i], Li)
+            np.testing.assert_allclose(ts[i, :Li], rts, rtol=1e-12, atol=0)
+            np.testing.assert_allclose(mb[i, :Li], rmb, rtol=1e-12, atol=0)
+            assert (ts[i, Li:] == 0).all()                      # rows beyond L[i] are left untouched
+        assert (sb.status == 0).all()
+
+
+def test_host_entry_point(orc, galv):
+    from paper_2504_03662_b200.search import HostSearch
+    for w, flags in ((inputs.config4(B=24), 1), (inputs.config2(), 3), (inputs.config0(), 2)):
+        hs = HostSearch(galv, w, flags)
+        res = hs.run()
+        res = {k: v.copy() for k, v in res.items()}
+        tq, mq, xq = oracle_tables(orc, w)
+        ref = oracle_search_many(orc, w, tq, mq, xq, list(range(w.B)))
+        for i in range(w.B):
+            Li = int(w.L[i])
+            assert res["opt_cost"][i] == ref[i]["opt_cost"] and (res["plan"][i, :Li] == ref[i]["plan"]).all()
+            assert res["status"][i] == ref[i]["status"] and res["mem_used"][i] == ref[i]["mem_used"]
+        again = hs.run()                                           # same arena, second call
+        assert (again["opt_cost"] == res["opt_cost"]).all() and (again["plan"] == res["plan"]).all()
+
+
+def test_boundary_errors(galv):
+    import ctypes as C
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    w = inputs.config0()
+    sb = SearchBuffers(galv, w, 1)
+    lib, h = galv.lib, galv.h
+    st = torch.cuda.current_stream().cuda_stream
+    p = lambda t: None if t is None else t.data_ptr()
+    ws_bytes = sb.workspace.numel()
+
+    def dp(shape, C_=sb.C, A_=None, ws=sb.workspace, nbytes=ws_bytes, L=sb.L):
+        return lib.galv_dp_search(h, C.byref(shape), p(L), p(sb.time_q), p(sb.mem_q), p(sb.trans_q), p(C_), p(A_),
+                                  p(sb.C_last), p(ws) if ws is not None else None, nbytes, p(sb.status), st)
+
+    assert dp(sb.shape) == gb.OK
+    assert dp(sb.shape, L=None) == gb.ERR_INVALID_ARG
+    assert dp(sb.shape, C_=None) == gb.ERR_INVALID_ARG                       # flag says full C
+    assert dp(gb.make_shape(1, 4, 6, 64, 0), C_=sb.C) == gb.ERR_INVALID_ARG  # table without its flag
+    assert dp(gb.make_shape(1, 4, 257, 64, 1)) == gb.ERR_INVALID_ARG         # S above the limit
+    assert dp(gb.make_shape(1, 4, 6, 64, 1, m_pitch=65)) == gb.ERR_INVALID_ARG
+    assert dp(gb.make_shape(1, 4, 6, 64, 1, m_pitch=64)) == gb.ERR_INVALID_ARG
+    assert dp(gb.make_shape(0, 4, 6, 64, 1)) == gb.ERR_INVALID_ARG
+    assert dp(sb.shape, ws=None) == gb.ERR_WORKSPACE
+    assert dp(sb.shape, nbytes=16) == gb.ERR_WORKSPACE
+    assert lib.galv_dp_workspace_bytes(h, C.byref(gb.make_shape(1, 4, 300, 64, 1))) == 0
+    assert b"workspace" in lib.galv_last_error(h)
+    assert lib.galv_strerror(gb.ERR_WORKSPACE) and lib.galv_strerror(-99)
+    # backtrack without any table to walk
+    rc = lib.galv_backtrack(h, C.byref(sb.shape), p(sb.L), p(sb.time_q), p(sb.mem_q), p(sb.trans_q), None, None,
+                            p(sb.C_last), None, p(sb.opt_cost), p(sb.plan), p(sb.mem_used), p(sb.status), st)
+    assert rc == gb.ERR_INVALID_ARG
+    # ... but the optimum alone is fine
+    rc = lib.galv_backtrack(h, C.byref(sb.shape), p(sb.L), p(sb.time_q), p(sb.mem_q), p(sb.trans_q), None, None,
+                            p(sb.C_last), None, p(sb.opt_cost), None, None, p(sb.status), st)
+    assert rc == gb.OK
+    torch.cuda.synchronize()
+    assert sb.opt_cost.item() == 7693
+    with pytest.raises(gb.GalvError):
+        galv.galv_dp_search(gb.make_shape(1, 4, 6, 64, 3), sb.L, sb.time_q, sb.mem_q, sb.trans_q, sb.C, None,
+                            sb.C_last, sb.workspace, sb.status)
+    h2 = C.c_void_p()
+    assert lib.galv_create(C.byref(h2), 9999) != gb.OK and not h2.value
+    torch.cuda.synchronize()                      # the context is still healthy
+    assert dp(sb.shape) == gb.OK
+
+
+def test_alu_probe_runs(galv):
+    rates = [galv.galv_probe_int_alu(k, 512) for k in (0, 1, 2)]
+    assert all(1e11 < r < 1e15 for r in rates), rates
