@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the strategy-search path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 3] [--impl reference]
+
+A step is one pass of the whole path over one batch of synthetic search
+instances: cost model -> validation -> layer-wise min-plus recurrence ->
+optimum -> plan backtrack.  Prints ONE JSON line (rank 0).
+
+Metric: DP cell updates per second (cells = sum_i L_i * (M+1) * S); searches/s
+and min-plus relaxations/s are reported beside it.  With N > 1 every rank runs
+its own batch of independent instances (no exchange on the data path; weak
+scaling); the time is the maximum over ranks.
+
+--impl reference times the CPU oracle (plain C, one instance per thread) on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2504_03662_b200 import inputs  # noqa: E402
+
+METRIC, UNIT = "dp_cell_updates_per_s", "cells/s"
+# Integer-ALU peak of one B200: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min
+# (one min-plus relaxation) per lane per clock.
+ALU_PEAK_GOPS = 148 * 64 * 1.965
+
+
+def workload_for(k: int, rank: int = 0, batch: int = 0, layers: int = 0):
+    w = inputs.CONFIGS[k]()
+    if batch or layers:
+        # trimmed copy of the workload (first `batch` instances, first `layers` layers) for profiler captures
+        w = w.take(slice(0, batch or w.B))
+        if layers and layers < w.Lmax:
+            w.Lmax = layers
+            w.L = np.minimum(w.L, layers).astype(np.int32)
+            if w.has_model:
+                w.layers = np.ascontiguousarray(w.layers[:, :layers])
+            else:
+                w.time_q = np.ascontiguousarray(w.time_q[:, :layers]); w.mem_q = np.ascontiguousarray(w.mem_q[:, :layers])
+        w.name += f"[B={w.B},L={w.Lmax}]"
+    if rank and w.has_model and k == 3:
+        # other ranks search other jittered instances of the same shape
+        u = inputs._unit(inputs.splitmix64(3 + 1000 * rank, 2 * w.B)).reshape(w.B, 2)
+        w.inst["flops_rate"] = 1e15 * (0.8 + 0.4 * u[:, 0])
+        w.inst["bw_tp"] = w.inst["bw_dp"] = 450e9 * (0.8 + 0.4 * u[:, 1])
+    return w
+
+
+# ------------------------------------------------------------------ CPU oracle legs
+
+def oracle_sample(w, max_layers: int, threads: int):
+    """First `threads` instances, first `max_layers` layers each: integer tables from the oracle's cost model."""
+    from oracle import oracle
+    k = min(threads, w.B)
+    items = []
+    for i in range(k):
+        Li = min(int(w.L[i]), max_layers)
+        if w.has_model:
+            _, _, tq, mq, xq = oracle.eval_costs(w.layers[0 if w.layers.shape[0] == 1 else i], w.strat, w.inst[i], Li)
+        else:
+            tq, mq, xq = w.time_q[i, :Li], w.mem_q[i, :Li], w.trans_q[i]
+        items.append((np.ascontiguousarray(tq), np.ascontiguousarray(mq), np.ascontiguousarray(xq)))
+    cells = sum(t.shape[0] for t, _, _ in items) * (w.M + 1) * w.S
+    return items, cells
+
+
+def oracle_run(w, items, threads: int) -> float:
+    """Seconds for the oracle to search every sampled instance (one instance per thread)."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import oracle
+
+    def one(it):
+        return oracle.search(it[0], it[1], it[2], w.M)["opt_cost"]
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(one, items))
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle
+    oracle.build()
+    w = workload_for(args.workload)
+    threads = min(os.cpu_count() or 1, w.B)
+    max_layers = max(2, min(w.Lmax, int(2.5e8 * 3.0 / ((w.M + 1) * w.S * w.S)) + 1))     # ~3 s of work per thread
+    items, cells = oracle_sample(w, max_layers, threads)
+    for _ in range(args.warmup):
+        oracle_run(w, items, threads)
+    ts = [oracle_run(w, items, threads) for _ in range(args.steps)]
+    t = sum(ts) / len(ts)
+    value = cells / t
+    sample = f"first {len(items)} instances x first {max_layers} layers per step, one instance per thread"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "Lmax": w.Lmax, "S": w.S, "M": w.M, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.rows, self.proc, self.uuid = [], None, uuid
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc:
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        reasons = [n for k, n in enumerate(names) if any(len(r) >= 7 and r[3 + k] == "Active" for r in self.rows)]
+        pw = [float(r[2]) for r in self.rows if len(r) >= 7 and r[2].replace(".", "").isdigit()]
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": float(self.rows[0][1]), "reasons": reasons,
+                "samples": len(sm), "power_w_max": max(pw) if pw else None}
+
+
+# ------------------------------------------------------------------ GPU arm
+
+def time_steps(torch, fn, steps, warmup, barrier):
+    """CUDA-event time of `steps` calls of fn on the current stream, in seconds (after warm-up, barriers both sides)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    return e0.elapsed_time(e1) * 1e-3
+
+
+def launches_per_step(w) -> int:
+    # cost + trans kernels, validate + schedule + base layer + (Lmax-1) layer kernels + finalize, backtrack
+    return (2 if w.has_model else 0) + 3 + (w.Lmax - 1) + 1 + 1
+
+
+def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):
+    from paper_2504_03662_b200.search import SearchBuffers
+    sb = SearchBuffers(galv, w, flags)
+    galv.galv_set_profiling(True)
+    t = time_steps(torch, sb.step, steps, warmup, barrier)
+    layer_ms = galv.galv_last_layer_loop_ms()                    # all layer launches of the last search, back to back
+    galv.galv_set_profiling(False)
+    res = sb.results()
+    out = {"seconds": t, "ms_per_step": t / steps * 1e3, "cells_per_s": w.cells * steps / t,
+           "relax_per_s": w.relaxations * steps / t, "searches_per_s": w.B * steps / t,
+           "layer_kernel_ms_avg": layer_ms / max(1, w.Lmax - 1), "layer_loop_ms": layer_ms,
+           "feasible": int((res["status"] == 0).sum()), "opt_cost_sum": int(res["opt_cost"][res["status"] == 0].sum())}
+    return sb, out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", type=int, default=3, help="workload index 0..4 (3: heterogeneous stack, the whole path)")
+    ap.add_argument("--impl", default="galv", choices=["galv", "reference"])
+    ap.add_argument("--no-others", action="store_true", help="skip the side measurements of the other workloads")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiler captures)")
+    ap.add_argument("--batch", type=int, default=0, help="trim the workload to its first instances (profiler captures)")
+    ap.add_argument("--layers", type=int, default=0, help="trim the workload to its first layers (profiler captures)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "galv" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import HostSearch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the search has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    galv = gb.Galv(local)
+    w = workload_for(args.workload, rank, args.batch, args.layers)
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", "")
+
+    with ClockSampler(uuid) as clk:
+        sb, r = bench_workload(torch, galv, w, args.steps, args.warmup, barrier)
+    t = max_over_ranks(r["seconds"])
+    clocks = clk.summary()
+    value = world * w.cells * args.steps / t
+    layer_s = r["layer_kernel_ms_avg"] * 1e-3
+    relax_per_launch = int((np.minimum(w.L, w.Lmax) - 1).clip(min=0).sum()) * (w.M + 1) * w.S * w.S / max(1, w.Lmax - 1)
+    achieved = relax_per_launch / layer_s / 1e9
+    del sb
+    torch.cuda.empty_cache()
+
+    # end to end through the host-buffer entry point: pinned host inputs -> device -> search -> host results
+    e2e = None
+    if not args.no_e2e:
+        hs = HostSearch(galv, w, gb.STORE_C_FULL)
+        for _ in range(args.warmup):
+            hs.run()
+        torch.cuda.synchronize(); barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            hs.run()
+        torch.cuda.synchronize(); barrier()
+        te = max_over_ranks(time.perf_counter() - t0)
+        e2e = {"value": world * w.cells * args.steps / te, "unit": UNIT, "ms_per_step": te / args.steps * 1e3,
+               "h2d_bytes_per_step": hs.h2d, "d2h_bytes_per_step": hs.d2h}
+        del hs
+        torch.cuda.empty_cache()
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": t / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "Lmax": w.Lmax, "S": w.S, "M": w.M, "per_gpu_batch": w.B,
+                   "tables": "full C kept (int32), plan re-derived along the path",
+                   "l2": "tables far larger than L2 (no flush needed)", "parallelism": f"instances x{world}"},
+        "searches_per_s": world * w.B * args.steps / t, "relaxations_per_s": world * w.relaxations * args.steps / t,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(w) * args.steps,
+        "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_GOPS, "unit": "G add-min/s",
+                     "frac": achieved / ALU_PEAK_GOPS, "traffic": None,
+                     "kernel": "layer_tiled_kernel", "launch_ms": r["layer_kernel_ms_avg"],
+                     "peak_source": "derived: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min per lane per clock"},
+    }
+
+    if rank == 0:
+        try:
+            line["roofline"]["probe_gops"] = {k: galv.galv_probe_int_alu(i, 4096) / 1e9
+                                              for i, k in enumerate(("fused_addmin", "add_then_min", "add_xor_2ops"))}
+        except gb.GalvError as e:      # diagnostic only
+            line["roofline"]["probe_gops"] = str(e)
+        # HBM side of the roofline: every table cell written once and read once by the next layer
+        from paper_2504_03662_b200.binding import make_shape
+        pitch = make_shape(w.B, w.Lmax, w.S, w.M).m_pitch
+        hbm_bytes = 2 * 4 * w.B * w.Lmax * w.S * pitch
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except OSError:
+            pass
+        hbm_gbs = peaks.get("hbm_gbs", 6650.0)
+        line["roofline"]["t_alu_ms"] = w.relaxations / (ALU_PEAK_GOPS * 1e9) * 1e3
+        line["roofline"]["t_hbm_ms"] = hbm_bytes / (hbm_gbs * 1e9) * 1e3
+        line["roofline"]["hbm_peak"] = f"{hbm_gbs} GB/s " + ("of measured" if peaks else "of fallback")
+        line["roofline"]["step_frac_of_bound"] = max(line["roofline"]["t_alu_ms"], line["roofline"]["t_hbm_ms"]) / (t / args.steps * 1e3)
+
+    if rank == 0 and world == 1 and not args.no_others:
+        others = {}
+        for k in (0, 1, 2, 4):
+            wk = workload_for(k)
+            sbk, rk = bench_workload(torch, galv, wk, max(5, args.steps // 2), 3, barrier)
+            o = {key: rk[key] for key in ("ms_per_step", "cells_per_s", "relax_per_s", "searches_per_s")}
+            o["alu_frac"] = rk["relax_per_s"] / (ALU_PEAK_GOPS * 1e9)
+            # the same step replayed from a CUDA graph (launch latency matters for the small workloads)
+            g = torch.cuda.CUDAGraph()
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                sbk.step()
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=s):
+                    sbk.step()
+                tg = time_steps(torch, g.replay, max(5, args.steps // 2), 3, barrier)
+            o["graph_ms_per_step"] = tg / max(5, args.steps // 2) * 1e3
+            others[wk.name] = o
+            del sbk, g
+            torch.cuda.empty_cache()
+        line["others"] = others
+
+    if rank == 0 and world == 1 and not args.no_cpu:
+        from oracle import oracle
+        oracle.build()
+        threads = min(os.cpu_count() or 1, w.B, 32)
+        max_layers = max(2, min(w.Lmax, int(2.5e8 * 10.0 / ((w.M + 1) * w.S * w.S)) + 1))   # ~10 s of work per thread
+        items, cells = oracle_sample(w, max_layers, threads)
+        tc = oracle_run(w, items, threads)
+        line["cpu_baseline"] = {"value": cells / tc, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": tc,
+                                "sample": f"first {len(items)} instances x first {max_layers} layers, one instance per thread"}
+    elif rank == 0:
+        line["cpu_baseline"] = None
+
+    if rank == 0:
+        print(json.dumps(line))
+    galv.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

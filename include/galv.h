@@ -194,6 +194,16 @@ int galv_search_host(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
  */
 int galv_probe_int_alu(galv_ctx* ctx, int kind, int iters, double* ops_per_s, void* stream);
 
+/*
+ * Timing hook for benchmarks (the paper has no counterpart).  While profiling is
+ * on, galv_dp_search records one CUDA event before its first layer launch and
+ * one after its last; galv_last_layer_loop_ms waits for the second and returns
+ * the milliseconds between them for the most recent search (host pointer).
+ * Leave it off when capturing a CUDA graph.
+ */
+int galv_set_profiling(galv_ctx* ctx, int on);
+int galv_last_layer_loop_ms(galv_ctx* ctx, float* ms);
+
 #ifdef __cplusplus
 }
 #endif

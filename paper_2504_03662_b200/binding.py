@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgalv.so"
 
 EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "galv_eval_costs",
            "galv_dp_workspace_bytes", "galv_dp_search", "galv_backtrack", "galv_search_host_arena_bytes",
-           "galv_search_host", "galv_probe_int_alu")
+           "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms")
 
 
 class galv_shape(C.Structure):
@@ -64,6 +64,8 @@ def load_library() -> C.CDLL:
     lib.galv_search_host_arena_bytes.restype = sz
     lib.galv_search_host.argtypes = [vp, shp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.galv_probe_int_alu.argtypes = [vp, C.c_int, C.c_int, C.POINTER(C.c_double), vp]
+    lib.galv_set_profiling.argtypes = [vp, C.c_int]
+    lib.galv_last_layer_loop_ms.argtypes = [vp, C.POINTER(C.c_float)]
     _lib = lib
     return lib
 
@@ -143,4 +145,12 @@ class Galv:
     def galv_probe_int_alu(self, kind: int, iters: int = 4096) -> float:
         out = C.c_double()
         self._check(self.lib.galv_probe_int_alu(self.h, kind, iters, C.byref(out), _stream()))
+        return out.value
+
+    def galv_set_profiling(self, on: bool):
+        self._check(self.lib.galv_set_profiling(self.h, int(on)))
+
+    def galv_last_layer_loop_ms(self) -> float:
+        out = C.c_float()
+        self._check(self.lib.galv_last_layer_loop_ms(self.h, C.byref(out)))
         return out.value

@@ -77,18 +77,32 @@ int galv_create(galv_ctx** out, int device_ordinal)
     ctx->num_sms = prop.multiProcessorCount;
     ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
     ctx->err[0] = 0;
+    ctx->profiling = 0;
+    ctx->ev_valid = 0;
+    ctx->ev0 = ctx->ev1 = nullptr;
     int cur = -1;
     cudaGetDevice(&cur);
     if (cur != device_ordinal) cudaSetDevice(device_ordinal);
     e = galv_dp_configure(ctx);
+    if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev0);
+    if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev1);
     if (cur >= 0 && cur != device_ordinal) cudaSetDevice(cur);
-    if (e != cudaSuccess) { delete ctx; return GALV_ERR_CUDA; }
+    if (e != cudaSuccess) {
+        if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+        if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+        delete ctx;
+        return GALV_ERR_CUDA;
+    }
     *out = ctx;
     return GALV_OK;
 }
 
 int galv_destroy(galv_ctx* ctx)
 {
+    if (ctx) {
+        if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+        if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+    }
     delete ctx;
     return GALV_OK;
 }
@@ -279,6 +293,22 @@ int galv_search_host(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, cons
     for (size_t i = 0; i < B; ++i)
         if (status[i] & GALV_STATUS_TIMEOUT) { set_err(ctx, "galv_search_host: device-side wait ran out"); return GALV_ERR_TIMEOUT; }
     return GALV_OK;
+}
+
+int galv_set_profiling(galv_ctx* ctx, int on)
+{
+    if (!ctx) return GALV_ERR_INVALID_ARG;
+    ctx->profiling = on != 0;
+    return GALV_OK;
+}
+
+int galv_last_layer_loop_ms(galv_ctx* ctx, float* ms)
+{
+    if (!ctx || !ms) return GALV_ERR_INVALID_ARG;
+    if (!ctx->ev_valid) { set_err(ctx, "galv_last_layer_loop_ms: no profiled search yet"); return GALV_ERR_INVALID_ARG; }
+    cudaError_t e = cudaEventSynchronize(ctx->ev1);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(ms, ctx->ev0, ctx->ev1);
+    return e == cudaSuccess ? GALV_OK : cuda_fail(ctx, "galv_last_layer_loop_ms", e);
 }
 
 int galv_probe_int_alu(galv_ctx* ctx, int kind, int iters, double* ops_per_s, void* stream)

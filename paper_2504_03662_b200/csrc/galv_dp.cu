@@ -477,7 +477,7 @@ cudaError_t galv_dp_configure(const galv_ctx* ctx)
     return e;
 }
 
-cudaError_t galv_dp_launch(const galv_ctx* ctx, const galv_shape* sh, const DpArgs& a, cudaStream_t st)
+cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a, cudaStream_t st)
 {
     cudaError_t e;
     const int B = a.B, Lmax = a.Lmax, S = a.S;
@@ -507,6 +507,7 @@ cudaError_t galv_dp_launch(const galv_ctx* ctx, const galv_shape* sh, const DpAr
     const bool reference = (sh->flags & GALV_KERNEL_REFERENCE) != 0;
     DpPlan pl;
     if (!reference && !galv_dp_make_plan(ctx, sh, &pl)) return cudaErrorInvalidConfiguration;
+    if (ctx->profiling) cudaEventRecord(ctx->ev0, st);
     for (int l = 1; l < Lmax; ++l) {
         if (reference) {
             const int mchunks = (a.m_pitch + 255) / 256;
@@ -517,6 +518,7 @@ cudaError_t galv_dp_launch(const galv_ctx* ctx, const galv_shape* sh, const DpAr
         }
         if (e != cudaSuccess) return e;
     }
+    if (ctx->profiling) { cudaEventRecord(ctx->ev1, st); ctx->ev_valid = 1; }
     finalize_kernel<<<(B + 255) / 256, 256, 0, st>>>(B, a.err, a.status);
     return cudaGetLastError();
 }

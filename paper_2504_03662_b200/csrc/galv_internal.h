@@ -11,6 +11,9 @@ struct galv_ctx {
     int device;
     int num_sms;
     int smem_optin;      // max dynamic shared memory per block (bytes)
+    int profiling;       // record ev0/ev1 around the layer launches
+    int ev_valid;        // ev0/ev1 have been recorded at least once
+    cudaEvent_t ev0, ev1;
     char err[512];
 };
 
@@ -53,7 +56,7 @@ WsLayout galv_ws_layout(const galv_shape* sh);
 
 bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* plan);
 cudaError_t galv_dp_configure(const galv_ctx* ctx);
-cudaError_t galv_dp_launch(const galv_ctx* ctx, const galv_shape* sh, const DpArgs& a, cudaStream_t st);
+cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a, cudaStream_t st);
 cudaError_t galv_backtrack_launch(const galv_shape* sh, const int32_t* L, const int32_t* time_q,
                                   const int32_t* mem_q, const int32_t* trans_q, const int32_t* C,
                                   const uint8_t* A, const int32_t* C_last, const int32_t* budget,
