@@ -390,12 +390,16 @@ __global__ void __launch_bounds__(512, 1) layer_tiled_kernel(const DpArgs a, con
                     const int mm = __ldg(a.mem_q + qrow + s);
                     const int lo = min(mm, M + 1);
                     const size_t o = (size_t)s * m_pitch;
-                    for (int m = lane; m < m_pitch; m += 32)
-                        if (m < lo || m > M) {
-                            out[o + m] = kInf;
-                            if (is_last) last[o + m] = kInf;
-                            if (ARG) aout[o + m] = 255;
-                        }
+                    for (int m = lane; m < lo; m += 32) {
+                        out[o + m] = kInf;
+                        if (is_last) last[o + m] = kInf;
+                        if (ARG) aout[o + m] = 255;
+                    }
+                    for (int m = M + 1 + lane; m < m_pitch; m += 32) {
+                        out[o + m] = kInf;
+                        if (is_last) last[o + m] = kInf;
+                        if (ARG) aout[o + m] = 255;
+                    }
                 }
             }
             cp_kc = 0;
