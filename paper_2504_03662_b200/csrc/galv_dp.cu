@@ -9,10 +9,10 @@
 // C[l][s][m'+mem(l,s)] = time(l,s) + G[s][m'].  So the kernel tiles like a
 // CUDA-core GEMM: an item is (instance, tile of m', block of s); warps own a
 // register tile of (TM x 32 columns) x (8 strategies); the previous layer's rows
-// are staged in shared memory by bulk async copies (TMA unit) and the S x S
-// transition rows by cp.async, double buffered over chunks of s'.  One fused
-// add-min instruction per relaxation; no tensor cores (min-plus is not a
-// multiply-add contraction).
+// and the matching rows of the S x S transition matrix are staged in shared memory
+// by bulk async copies (TMA unit) issued by a producer warp, in a multi-stage
+// mbarrier pipeline over chunks of s'.  One fused add-min instruction per
+// relaxation; no tensor cores (min-plus is not a multiply-add contraction).
 //
 // One launch per layer (a layer needs all of the previous one); launches are
 // plain stream work, so a caller may capture the whole search in a CUDA graph.
@@ -36,6 +36,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -57,14 +60,6 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void cp_async4(void* dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
 // ---------------------------------------------------------------- validation / schedule
 
@@ -191,221 +186,233 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 }
 
 // ---------------------------------------------------------------- tiled layer kernel
+//
+// Work items are (instance, m'-tile, s-block); every CTA owns a contiguous run of them, so
+// consecutive items mostly share the instance (its trans rows stay in L2).  Warp roles:
+//   warp NC (producer): for every chunk (item, k-chunk of s') waits for a free stage, then
+//       bulk-copies KS rows of the previous layer's slice and the matching rows of trans into it;
+//       also writes the cells no column maps to (m < mem(l,s)) and the pad columns;
+//   warps 0..NC-1 (consumers): warp (ms, sg) keeps a TM x 8 register tile per lane
+//       (columns m' = tile + ms*32*TM + j*32 + lane, strategies sg*8 .. sg*8+7), waits for the
+//       stage, runs one fused add-min per relaxation, releases the stage, and after the last
+//       chunk stores column m' of strategy s at m' + mem(l,s).
+// Stages are handed over with mbarriers (full: bytes landed; empty: every consumer warp done),
+// so there is no block-wide barrier in the loop.  Every wait is bounded.
 
-struct Item { int i, mt, sb; };
+constexpr int kMaxStages = 4;
 
-__device__ __forceinline__ Item decode_item(long long item, const DpPlan& pl, const int32_t* __restrict__ order) {
+struct ItemPos { int oi, mt, sb; };
+
+__device__ __forceinline__ ItemPos item_at(long long item, const DpPlan& pl) {
     const int per = pl.ntiles_m * pl.nsb;
-    const int oi = (int)(item / per);
-    const int r = (int)(item - (long long)oi * per);
-    Item it;
-    it.i = order[oi];
-    it.mt = r / pl.nsb;
-    it.sb = r - it.mt * pl.nsb;
-    return it;
+    ItemPos p;
+    p.oi = (int)(item / per);
+    const int r = (int)(item - (long long)p.oi * per);
+    p.mt = r / pl.nsb;
+    p.sb = r - p.mt * pl.nsb;
+    return p;
+}
+__device__ __forceinline__ void item_next(ItemPos& p, const DpPlan& pl) {
+    if (++p.sb == pl.nsb) { p.sb = 0; if (++p.mt == pl.ntiles_m) { p.mt = 0; ++p.oi; } }
 }
 
 template <int TM, bool ARG>
-__global__ void __launch_bounds__(512, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l)
+__global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[2];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nthreads = blockDim.x;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
-    const int TMB = pl.tmb, SB = pl.sb, KS = pl.ks, NKC = pl.nkc;
-    const int sg = warp % pl.nsg, ms = warp / pl.nsg;
+    const int TMB = pl.tmb, SB = pl.sb, KS = pl.ks, NKC = pl.nkc, NST = pl.nst;
+    const int NC = pl.nsg * pl.nms;                       // consumer warps
 
     const long long nitems = (long long)a.nactive[l] * pl.ntiles_m * pl.nsb;
-    if ((long long)blockIdx.x >= nitems) return;
+    const long long it0 = nitems * blockIdx.x / gridDim.x, it1 = nitems * (blockIdx.x + 1) / gridDim.x;
+    if (it0 >= it1) return;
 
     int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
     const int stage_elems = KS * (TMB + SB);
 
     if (tid == 0) {
-        mbar_init(&full_bar[0], 1);
-        mbar_init(&full_bar[1], 1);
+        for (int k = 0; k < NST; ++k) { mbar_init(&full_bar[k], 1); mbar_init(&empty_bar[k], NC); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
     const size_t slice = (size_t)S * m_pitch;
-    const bool vec16 = (S & 3) == 0;
+    ItemPos pos = item_at(it0, pl);
 
-    // Stage one chunk (item, kc): rows k0..k0+kn of the previous layer's slice, columns
-    // [m0, m0+w), by bulk copies from warp 0; the matching rows of trans by cp.async from all.
-    auto issue_load = [&](long long item, int kc, int st) {
-        const Item it = decode_item(item, pl, a.order);
-        const int m0 = it.mt * TMB;
-        const int w = min(TMB, m_pitch - m0);
-        const int k0 = kc * KS;
-        const int kn = min(KS, S - k0);
-        const int sb0 = it.sb * SB;
-        int32_t* cs = stage0 + st * stage_elems;
-        int32_t* ts = cs + KS * TMB;
-        const int32_t* prev = (a.C ? a.C + ((size_t)it.i * a.Lmax + (l - 1)) * slice
-                                   : a.roll + ((size_t)((l - 1) & 1) * a.B + it.i) * slice)
-                              + (size_t)k0 * m_pitch + m0;
-        if (warp == 0) {
-            if (lane == 0) mbar_expect_tx(&full_bar[st], (uint32_t)kn * w * 4u);
-            __syncwarp();
-            for (int r = lane; r < kn; r += 32)
-                bulk_g2s(cs + r * TMB, prev + (size_t)r * m_pitch, (uint32_t)w * 4u, &full_bar[st]);
-        }
-        const int32_t* T = a.trans_q + (size_t)it.i * S * S + (size_t)k0 * S + sb0;
-        if (vec16) {
-            const int q = SB >> 2;
-            for (int e = tid; e < kn * q; e += nthreads) {
-                const int r = e / q, c = (e - r * q) << 2;
-                if (sb0 + c < S) cp_async16(ts + r * SB + c, T + (size_t)r * S + c);
+    if (warp == NC) {
+        // ------------------------------------------------------------ producer
+        const bool bulk_t = (S & 3) == 0;                 // trans rows 16-byte aligned
+        int n = 0;                                        // chunk counter
+        for (long long item = it0; item < it1; ++item, item_next(pos, pl)) {
+            const int i = a.order[pos.oi];
+            const int m0 = pos.mt * TMB;
+            const int w = min(TMB, m_pitch - m0);
+            const int sb0 = pos.sb * SB;
+            const int sbw = min(SB, S - sb0);             // strategies of this block that exist
+            const int32_t* prev = (a.C ? a.C + ((size_t)i * a.Lmax + (l - 1)) * slice
+                                       : a.roll + ((size_t)((l - 1) & 1) * a.B + i) * slice) + m0;
+            const int32_t* T = a.trans_q + (size_t)i * S * S + sb0;
+            for (int kc = 0; kc < NKC; ++kc, ++n) {
+                const int st = n % NST;
+                if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+                const int k0 = kc * KS;
+                const int kn = min(KS, S - k0);
+                int32_t* cs = stage0 + st * stage_elems;
+                int32_t* ts = cs + KS * TMB;
+                if (!bulk_t) {
+                    // unaligned trans rows: plain copies by this warp, published by the arrive below
+                    for (int e = lane; e < kn * sbw; e += 32) {
+                        const int r = e / sbw, c = e - r * sbw;
+                        ts[r * SB + c] = __ldg(T + (size_t)(k0 + r) * S + c);
+                    }
+                    __syncwarp();
+                }
+                if (lane == 0)
+                    mbar_expect_tx(&full_bar[st], (uint32_t)kn * (uint32_t)(w + (bulk_t ? sbw : 0)) * 4u);
+                __syncwarp();
+                for (int r = lane; r < kn; r += 32) {
+                    bulk_g2s(cs + r * TMB, prev + (size_t)(k0 + r) * m_pitch, (uint32_t)w * 4u, &full_bar[st]);
+                    if (bulk_t) bulk_g2s(ts + r * SB, T + (size_t)(k0 + r) * S, (uint32_t)sbw * 4u, &full_bar[st]);
+                }
             }
-        } else {
-            for (int e = tid; e < kn * SB; e += nthreads) {
-                const int r = e / SB, c = e - r * SB;
-                if (sb0 + c < S) cp_async4(ts + r * SB + c, T + (size_t)r * S + c);
+            if (pos.mt == 0) {
+                // Cells no column maps to: m < mem(l,s), and the pad columns.
+                const bool is_last = (a.L[i] == l + 1);
+                int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
+                int32_t* last = a.C_last + (size_t)i * slice;
+                uint8_t* aout = ARG ? a.A + ((size_t)i * a.Lmax + l) * slice : nullptr;
+                const size_t qrow = ((size_t)i * a.Lmax + l) * S;
+                for (int s = sb0; s < sb0 + sbw; ++s) {
+                    const int lo = min(__ldg(a.mem_q + qrow + s), M + 1);
+                    const size_t o = (size_t)s * m_pitch;
+                    for (int m = lane; m < lo + (m_pitch - M - 1); m += 32) {
+                        const int mm = m < lo ? m : m - lo + M + 1;
+                        out[o + mm] = kInf;
+                        if (is_last) last[o + mm] = kInf;
+                        if (ARG) aout[o + mm] = 255;
+                    }
+                }
             }
         }
-        cp_async_commit();
-    };
+        return;
+    }
+    if (warp > NC) return;
 
-    long long ld_item = blockIdx.x; int ld_kc = 0;       // load cursor
-    long long cp_item = blockIdx.x; int cp_kc = 0;       // compute cursor
-    issue_load(ld_item, ld_kc, 0);
-    if (++ld_kc == NKC) { ld_kc = 0; ld_item += gridDim.x; }
-
+    // ---------------------------------------------------------------- consumers
+    const int sg = warp % pl.nsg, ms = warp / pl.nsg;
     int acc[TM][TS];
     int arg[ARG ? TM : 1][ARG ? TS : 1];
     (void)arg;
-
-    for (int iter = 0; cp_item < nitems; ++iter) {
-        const int st = iter & 1;
-        cp_async_wait_all();
-        if (!mbar_wait(&full_bar[st], (iter >> 1) & 1)) {
-            // Give up cleanly: flag the error; a second bounded wait lets copies in flight land.
-            if (tid == 0) atomicExch(a.err, 1);
-            mbar_wait(&full_bar[st], (iter >> 1) & 1);
-            return;
-        }
-        __syncthreads();      // trans rows visible to all; everyone is done with the other stage
-        if (ld_item < nitems) {
-            issue_load(ld_item, ld_kc, st ^ 1);
-            if (++ld_kc == NKC) { ld_kc = 0; ld_item += gridDim.x; }
-        }
-
-        const Item it = decode_item(cp_item, pl, a.order);
-        const int m0 = it.mt * TMB;
-        const int k0 = cp_kc * KS;
-        const int kn = min(KS, S - k0);
+    int n = 0;
+    for (long long item = it0; item < it1; ++item, item_next(pos, pl)) {
+        const int m0 = pos.mt * TMB;
         const int mw = m0 + ms * (32 * TM);                 // first column of this warp
         // 32-column groups of this warp that hold at least one column <= M
         const int nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
-
-        if (cp_kc == 0) {
 #pragma unroll
-            for (int j = 0; j < TM; ++j)
-#pragma unroll
-                for (int u = 0; u < TS; ++u) {
-                    acc[j][u] = 0x7fffffff;
-                    if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = 255;
-                }
-        }
-
-        const int32_t* cs = stage0 + st * stage_elems + ms * (32 * TM) + lane;
-        const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
-
-        if (nj == TM) {
-#pragma unroll 2
-            for (int k = 0; k < kn; ++k) {
-                int c[TM];
-#pragma unroll
-                for (int j = 0; j < TM; ++j) c[j] = cs[k * TMB + j * 32];
-                const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
-                const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
-                const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-#pragma unroll
-                for (int j = 0; j < TM; ++j)
-#pragma unroll
-                    for (int u = 0; u < TS; ++u) {
-                        if (ARG) {
-                            const int cand = c[j] + t[u];
-                            if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
-                        } else {
-                            acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
-                        }
-                    }
-            }
-        } else if (nj > 0) {
-            // ragged last tile: only the first nj column groups carry work
-            for (int k = 0; k < kn; ++k) {
-                const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
-                const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
-                const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-#pragma unroll
-                for (int j = 0; j < TM; ++j)
-                    if (j < nj) {
-                        const int c = cs[k * TMB + j * 32];
-#pragma unroll
-                        for (int u = 0; u < TS; ++u) {
-                            const int cand = c + t[u];
-                            if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
-                        }
-                    }
-            }
-        }
-
-        if (cp_kc == NKC - 1) {
-            // Epilogue: column m' of strategy s lands at m = m' + mem(l,s).
-            const int i = it.i;
-            const bool is_last = (a.L[i] == l + 1);
-            int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
-            int32_t* last = a.C_last + (size_t)i * slice;
-            uint8_t* aout = ARG ? a.A + ((size_t)i * a.Lmax + l) * slice : nullptr;
-            const size_t qrow = ((size_t)i * a.Lmax + l) * S;
-            const int sb0 = it.sb * SB;
+        for (int j = 0; j < TM; ++j)
 #pragma unroll
             for (int u = 0; u < TS; ++u) {
-                const int s = sb0 + sg * TS + u;
+                acc[j][u] = 0x7fffffff;
+                if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = 255;
+            }
+        for (int kc = 0; kc < NKC; ++kc, ++n) {
+            const int st = n % NST;
+            if (!mbar_wait(&full_bar[st], (n / NST) & 1)) {
+                if (lane == 0) atomicExch(a.err, 1);
+                return;
+            }
+            const int k0 = kc * KS;
+            const int kn = min(KS, S - k0);
+            const int32_t* cs = stage0 + st * stage_elems + ms * (32 * TM) + lane;
+            const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
+            if (nj == TM) {
+#pragma unroll 4
+                for (int k = 0; k < kn; ++k) {
+                    int c[TM];
+#pragma unroll
+                    for (int j = 0; j < TM; ++j) c[j] = cs[k * TMB + j * 32];
+                    const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
+                    const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
+                    const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                    for (int j = 0; j < TM; ++j)
+#pragma unroll
+                        for (int u = 0; u < TS; ++u) {
+                            if (ARG) {
+                                const int cand = c[j] + t[u];
+                                if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
+                            } else {
+                                acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                            }
+                        }
+                }
+            } else if (nj > 0) {
+                // ragged last tile: only the first nj column groups carry work
+                for (int k = 0; k < kn; ++k) {
+                    const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
+                    const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
+                    const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                    for (int j = 0; j < TM; ++j)
+                        if (j < nj) {
+                            const int c = cs[k * TMB + j * 32];
+#pragma unroll
+                            for (int u = 0; u < TS; ++u) {
+                                const int cand = c + t[u];
+                                if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
+                            }
+                        }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[st]);      // this warp is done reading the stage
+        }
+
+        // Epilogue: column m' of strategy s lands at m = m' + mem(l,s).
+        if (nj > 0) {
+            const int i = a.order[pos.oi];
+            const bool is_last = (a.L[i] == l + 1);
+            int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
+            const size_t qrow = ((size_t)i * a.Lmax + l) * S;
+            const int s0 = pos.sb * SB + sg * TS;
+#pragma unroll
+            for (int u = 0; u < TS; ++u) {
+                const int s = s0 + u;
                 if (s < S) {
                     const int mm = __ldg(a.mem_q + qrow + s);
                     const int tt = __ldg(a.time_q + qrow + s);
+                    const int lim = M - mm - mw - lane;          // column group j is stored iff j*32 <= lim
+                    const size_t o = (size_t)s * m_pitch + (size_t)(mm + mw + lane);
+                    int32_t* po = out + o;
 #pragma unroll
                     for (int j = 0; j < TM; ++j) {
-                        const int mp = mw + j * 32 + lane;
-                        if (j < nj && mp <= M && mm <= M - mp) {
-                            const size_t o = (size_t)s * m_pitch + (mp + mm);
-                            const int g = acc[j][u];
-                            const int v = g >= kInf ? kInf : g + tt;
-                            out[o] = v;
-                            if (is_last) last[o] = v;
-                            if (ARG) aout[o] = (uint8_t)(g >= kInf ? 255 : arg[ARG ? j : 0][ARG ? u : 0]);
-                        }
+                        // finite sums stay below kInf; min(g, kInf) + tt cannot wrap
+                        const int v = __viaddmin_s32(min(acc[j][u], kInf), tt, kInf);
+                        if (j * 32 <= lim) po[j * 32] = v;
+                    }
+                    if (is_last) {
+                        int32_t* pl2 = a.C_last + (size_t)i * slice + o;
+#pragma unroll
+                        for (int j = 0; j < TM; ++j)
+                            if (j * 32 <= lim) pl2[j * 32] = __viaddmin_s32(min(acc[j][u], kInf), tt, kInf);
+                    }
+                    if (ARG) {
+                        uint8_t* pa = a.A + ((size_t)i * a.Lmax + l) * slice + o;
+#pragma unroll
+                        for (int j = 0; j < TM; ++j)
+                            if (j * 32 <= lim) pa[j * 32] = (uint8_t)(acc[j][u] >= kInf ? 255 : arg[ARG ? j : 0][ARG ? u : 0]);
                     }
                 }
             }
-            if (it.mt == 0) {
-                // Cells no column maps to: m < mem(l,s), and the pad columns.
-                const int nw = nthreads >> 5;
-                for (int s = sb0 + warp; s < min(S, sb0 + SB); s += nw) {
-                    const int mm = __ldg(a.mem_q + qrow + s);
-                    const int lo = min(mm, M + 1);
-                    const size_t o = (size_t)s * m_pitch;
-                    for (int m = lane; m < lo; m += 32) {
-                        out[o + m] = kInf;
-                        if (is_last) last[o + m] = kInf;
-                        if (ARG) aout[o + m] = 255;
-                    }
-                    for (int m = M + 1 + lane; m < m_pitch; m += 32) {
-                        out[o + m] = kInf;
-                        if (is_last) last[o + m] = kInf;
-                        if (ARG) aout[o + m] = 255;
-                    }
-                }
-            }
-            cp_kc = 0;
-            cp_item += gridDim.x;
-        } else {
-            ++cp_kc;
         }
     }
 }
@@ -456,17 +463,22 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     pl->nms = 16 / pl->nsg;
     if (pl->nms < 1) pl->nms = 1;
     pl->tmb = pl->nms * 32 * pl->tm;
-    pl->threads = pl->nsg * pl->nms * 32;
-    // two stages of ks * (tmb + sb) ints must fit the opt-in shared memory
-    const int budget = (ctx->smem_optin - 1024) / 2;
-    int ks = budget / ((pl->tmb + pl->sb) * 4);
+    pl->threads = (pl->nsg * pl->nms + 1) * 32;           // consumer warps + the producer warp
+    // stages of ks * (tmb + sb) ints: aim at <= 40 KB each, 2..4 of them in the opt-in shared memory
+    const int avail = ctx->smem_optin - 2048;
+    const int row = (pl->tmb + pl->sb) * 4;
+    int ks = (40 * 1024) / row;
     if (ks > S) ks = S;
-    if (ks > 64) ks = 64;
-    if (ks < 1) return false;
+    if (ks >= 8) ks &= ~7;
+    if (ks < 1) ks = 1;
+    int nst = avail / (ks * row);
+    if (nst > kMaxStages) nst = kMaxStages;
+    if (nst < 2) return false;
     pl->ks = ks;
+    pl->nst = nst;
     pl->nkc = (S + ks - 1) / ks;
     pl->ntiles_m = (sh->M + 1 + pl->tmb - 1) / pl->tmb;
-    pl->smem = 2 * ks * (pl->tmb + pl->sb) * 4;
+    pl->smem = nst * ks * row;
     const long long items = (long long)sh->B * pl->ntiles_m * pl->nsb;
     pl->grid = (int)(items < ctx->num_sms ? items : ctx->num_sms);
     return true;
@@ -475,9 +487,9 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
 cudaError_t galv_dp_configure(const galv_ctx* ctx)
 {
     cudaError_t e;
-    e = cudaFuncSetAttribute(layer_tiled_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 1024);
+    e = cudaFuncSetAttribute(layer_tiled_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 2048);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(layer_tiled_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 1024);
+    e = cudaFuncSetAttribute(layer_tiled_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 2048);
     return e;
 }
 

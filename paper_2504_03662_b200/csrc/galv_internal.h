@@ -26,9 +26,10 @@ struct DpPlan {
     int nms;       // warps along m
     int tmb;       // budget columns per item = nms * 32 * tm
     int ks;        // previous-layer strategies staged per pipeline stage
-    int nkc;       // stages per item = ceil(S / ks)
+    int nkc;       // chunks per item = ceil(S / ks)
+    int nst;       // pipeline stages in shared memory
     int ntiles_m;  // ceil((M+1) / tmb)
-    int threads;   // nsg * nms * 32
+    int threads;   // (nsg * nms + 1) * 32: consumer warps and one producer warp
     int smem;      // dynamic shared memory bytes
     int grid;      // resident CTAs
 };
