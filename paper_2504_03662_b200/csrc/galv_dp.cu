@@ -216,17 +216,24 @@ __device__ __forceinline__ void item_next(ItemPos& p, const DpPlan& pl) {
     if (++p.sb == pl.nsb) { p.sb = 0; if (++p.mt == pl.ntiles_m) { p.mt = 0; ++p.oi; } }
 }
 
-template <int TM, bool ARG>
-__global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l)
+// Shared memory: NST stages of [KS][TMB] previous-layer values + [KS][SB] trans values, then per
+// stage a small record the producer fills for the item whose last chunk sits in that stage:
+// mem(l,s) and time(l,s) of the s-block, the instance index and whether l is its last layer.
+template <int TM, int NSG, int NMS, bool ARG>
+__global__ void __launch_bounds__((NSG * NMS + 1) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l)
 {
+    constexpr int NC = NSG * NMS;                         // consumer warps
+    constexpr int SB = NSG * TS;                          // strategies per item
+    constexpr int TMB = NMS * 32 * TM;                    // columns per item
+    constexpr int META = 2 * SB + 4;
+
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
-    const int TMB = pl.tmb, SB = pl.sb, KS = pl.ks, NKC = pl.nkc, NST = pl.nst;
-    const int NC = pl.nsg * pl.nms;                       // consumer warps
+    const int KS = pl.ks, NKC = pl.nkc, NST = pl.nst;
 
     const long long nitems = (long long)a.nactive[l] * pl.ntiles_m * pl.nsb;
     const long long it0 = nitems * blockIdx.x / gridDim.x, it1 = nitems * (blockIdx.x + 1) / gridDim.x;
@@ -234,6 +241,7 @@ __global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, con
 
     int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
     const int stage_elems = KS * (TMB + SB);
+    int32_t* const meta0 = stage0 + NST * stage_elems;
 
     if (tid == 0) {
         for (int k = 0; k < NST; ++k) { mbar_init(&full_bar[k], 1); mbar_init(&empty_bar[k], NC); }
@@ -254,6 +262,8 @@ __global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, con
             const int w = min(TMB, m_pitch - m0);
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
+            const bool is_last = (a.L[i] == l + 1);
+            const size_t qrow = ((size_t)i * a.Lmax + l) * S;
             const int32_t* prev = (a.C ? a.C + ((size_t)i * a.Lmax + (l - 1)) * slice
                                        : a.roll + ((size_t)((l - 1) & 1) * a.B + i) * slice) + m0;
             const int32_t* T = a.trans_q + (size_t)i * S * S + sb0;
@@ -273,8 +283,16 @@ __global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, con
                         const int r = e / sbw, c = e - r * sbw;
                         ts[r * SB + c] = __ldg(T + (size_t)(k0 + r) * S + c);
                     }
-                    __syncwarp();
                 }
+                if (kc == NKC - 1) {
+                    int32_t* meta = meta0 + st * META;
+                    for (int c = lane; c < sbw; c += 32) {
+                        meta[c] = __ldg(a.mem_q + qrow + sb0 + c);
+                        meta[SB + c] = __ldg(a.time_q + qrow + sb0 + c);
+                    }
+                    if (lane == 0) { meta[2 * SB] = i; meta[2 * SB + 1] = is_last; }
+                }
+                __syncwarp();
                 if (lane == 0)
                     mbar_expect_tx(&full_bar[st], (uint32_t)kn * (uint32_t)(w + (bulk_t ? sbw : 0)) * 4u);
                 __syncwarp();
@@ -285,11 +303,9 @@ __global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, con
             }
             if (pos.mt == 0) {
                 // Cells no column maps to: m < mem(l,s), and the pad columns.
-                const bool is_last = (a.L[i] == l + 1);
                 int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
                 int32_t* last = a.C_last + (size_t)i * slice;
                 uint8_t* aout = ARG ? a.A + ((size_t)i * a.Lmax + l) * slice : nullptr;
-                const size_t qrow = ((size_t)i * a.Lmax + l) * S;
                 for (int s = sb0; s < sb0 + sbw; ++s) {
                     const int lo = min(__ldg(a.mem_q + qrow + s), M + 1);
                     const size_t o = (size_t)s * m_pitch;
@@ -307,23 +323,23 @@ __global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, con
     if (warp > NC) return;
 
     // ---------------------------------------------------------------- consumers
-    const int sg = warp % pl.nsg, ms = warp / pl.nsg;
+    const int sg = warp % NSG, ms = warp / NSG;
     int acc[TM][TS];
     int arg[ARG ? TM : 1][ARG ? TS : 1];
     (void)arg;
     int n = 0;
     for (long long item = it0; item < it1; ++item, item_next(pos, pl)) {
-        const int m0 = pos.mt * TMB;
-        const int mw = m0 + ms * (32 * TM);                 // first column of this warp
+        const int mw = pos.mt * TMB + ms * (32 * TM);       // first column of this warp
         // 32-column groups of this warp that hold at least one column <= M
         const int nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
 #pragma unroll
         for (int j = 0; j < TM; ++j)
 #pragma unroll
             for (int u = 0; u < TS; ++u) {
-                acc[j][u] = 0x7fffffff;
+                acc[j][u] = kInf;                            // min over candidates never exceeds kInf
                 if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = 255;
             }
+        int mm[TS], tt[TS], inst = 0, is_last = 0;
         for (int kc = 0; kc < NKC; ++kc, ++n) {
             const int st = n % NST;
             if (!mbar_wait(&full_bar[st], (n / NST) & 1)) {
@@ -335,25 +351,46 @@ __global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, con
             const int32_t* cs = stage0 + st * stage_elems + ms * (32 * TM) + lane;
             const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
             if (nj == TM) {
-#pragma unroll 4
-                for (int k = 0; k < kn; ++k) {
-                    int c[TM];
+                int k = 0;
+                for (; k + 4 <= kn; k += 4) {
 #pragma unroll
-                    for (int j = 0; j < TM; ++j) c[j] = cs[k * TMB + j * 32];
-                    const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
-                    const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
+                    for (int kk = 0; kk < 4; ++kk) {
+                        int c[TM];
+#pragma unroll
+                        for (int j = 0; j < TM; ++j) c[j] = cs[kk * TMB + j * 32];
+                        const int4 t0 = *reinterpret_cast<const int4*>(ts + kk * SB);
+                        const int4 t1 = *reinterpret_cast<const int4*>(ts + kk * SB + 4);
+                        const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                        for (int j = 0; j < TM; ++j)
+#pragma unroll
+                            for (int u = 0; u < TS; ++u) {
+                                if (ARG) {
+                                    const int cand = c[j] + t[u];
+                                    if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k + kk; }
+                                } else {
+                                    acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                                }
+                            }
+                    }
+                    cs += 4 * TMB;
+                    ts += 4 * SB;
+                }
+                for (; k < kn; ++k) {
+                    const int4 t0 = *reinterpret_cast<const int4*>(ts);
+                    const int4 t1 = *reinterpret_cast<const int4*>(ts + 4);
                     const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
 #pragma unroll
-                    for (int j = 0; j < TM; ++j)
+                    for (int j = 0; j < TM; ++j) {
+                        const int c = cs[j * 32];
 #pragma unroll
                         for (int u = 0; u < TS; ++u) {
-                            if (ARG) {
-                                const int cand = c[j] + t[u];
-                                if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
-                            } else {
-                                acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
-                            }
+                            const int cand = c + t[u];
+                            if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
                         }
+                    }
+                    cs += TMB;
+                    ts += SB;
                 }
             } else if (nj > 0) {
                 // ragged last tile: only the first nj column groups carry work
@@ -373,37 +410,48 @@ __global__ void __launch_bounds__(544, 1) layer_tiled_kernel(const DpArgs a, con
                         }
                 }
             }
+            if (kc == NKC - 1) {
+                // the item's record must be read before the stage is handed back
+                const int32_t* meta = meta0 + st * META;
+                const int4 m0v = *reinterpret_cast<const int4*>(meta + sg * TS);
+                const int4 m1v = *reinterpret_cast<const int4*>(meta + sg * TS + 4);
+                const int4 t0v = *reinterpret_cast<const int4*>(meta + SB + sg * TS);
+                const int4 t1v = *reinterpret_cast<const int4*>(meta + SB + sg * TS + 4);
+                mm[0] = m0v.x; mm[1] = m0v.y; mm[2] = m0v.z; mm[3] = m0v.w; mm[4] = m1v.x; mm[5] = m1v.y; mm[6] = m1v.z; mm[7] = m1v.w;
+                tt[0] = t0v.x; tt[1] = t0v.y; tt[2] = t0v.z; tt[3] = t0v.w; tt[4] = t1v.x; tt[5] = t1v.y; tt[6] = t1v.z; tt[7] = t1v.w;
+                inst = meta[2 * SB];
+                is_last = meta[2 * SB + 1];
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);      // this warp is done reading the stage
         }
 
         // Epilogue: column m' of strategy s lands at m = m' + mem(l,s).
         if (nj > 0) {
-            const int i = a.order[pos.oi];
-            const bool is_last = (a.L[i] == l + 1);
+            const int i = inst;
             int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
-            const size_t qrow = ((size_t)i * a.Lmax + l) * S;
             const int s0 = pos.sb * SB + sg * TS;
+            const int base = M - mw - lane;                  // group j of strategy u is stored iff j*32 + mem <= base
 #pragma unroll
             for (int u = 0; u < TS; ++u) {
-                const int s = s0 + u;
-                if (s < S) {
-                    const int mm = __ldg(a.mem_q + qrow + s);
-                    const int tt = __ldg(a.time_q + qrow + s);
-                    const int lim = M - mm - mw - lane;          // column group j is stored iff j*32 <= lim
-                    const size_t o = (size_t)s * m_pitch + (size_t)(mm + mw + lane);
+                if (s0 + u < S) {
+                    const int lim = base - mm[u];
+                    const size_t o = (size_t)(s0 + u) * m_pitch + (size_t)(mm[u] + mw + lane);
                     int32_t* po = out + o;
+                    // finite sums stay below kInf and acc <= kInf, so acc + time cannot wrap
+                    if (__all_sync(0xffffffffu, lim >= (TM - 1) * 32)) {
 #pragma unroll
-                    for (int j = 0; j < TM; ++j) {
-                        // finite sums stay below kInf; min(g, kInf) + tt cannot wrap
-                        const int v = __viaddmin_s32(min(acc[j][u], kInf), tt, kInf);
-                        if (j * 32 <= lim) po[j * 32] = v;
+                        for (int j = 0; j < TM; ++j) po[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < TM; ++j)
+                            if (j * 32 <= lim) po[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
                     }
                     if (is_last) {
                         int32_t* pl2 = a.C_last + (size_t)i * slice + o;
 #pragma unroll
                         for (int j = 0; j < TM; ++j)
-                            if (j * 32 <= lim) pl2[j * 32] = __viaddmin_s32(min(acc[j][u], kInf), tt, kInf);
+                            if (j * 32 <= lim) pl2[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
                     }
                     if (ARG) {
                         uint8_t* pa = a.A + ((size_t)i * a.Lmax + l) * slice + o;
@@ -425,11 +473,30 @@ __global__ void finalize_kernel(int B, const int32_t* err, int32_t* status)
         status[i] |= GALV_STATUS_TIMEOUT;
 }
 
-template <int TM, bool ARG>
-cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st)
+template <int TM, int NSG, int NMS, bool ARG>
+cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st, bool configure)
 {
-    layer_tiled_kernel<TM, ARG><<<pl.grid, pl.threads, pl.smem, st>>>(a, pl, l);
+    auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG>;
+    if (configure) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+    kern<<<pl.grid, (NSG * NMS + 1) * 32, pl.smem, st>>>(a, pl, l);
     return cudaGetLastError();
+}
+
+// nsg warps along s, 16/nsg (rounded down) along m: one instantiation per s-block width.
+template <bool ARG>
+cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st, bool configure)
+{
+    switch (pl.nsg) {
+    case 1: return launch_one<4, 1, 16, ARG>(a, pl, l, st, configure);
+    case 2: return launch_one<4, 2, 8, ARG>(a, pl, l, st, configure);
+    case 3: return launch_one<4, 3, 5, ARG>(a, pl, l, st, configure);
+    case 4: return launch_one<4, 4, 4, ARG>(a, pl, l, st, configure);
+    case 5: return launch_one<4, 5, 3, ARG>(a, pl, l, st, configure);
+    case 6: return launch_one<4, 6, 2, ARG>(a, pl, l, st, configure);
+    case 7: return launch_one<4, 7, 2, ARG>(a, pl, l, st, configure);
+    case 8: return launch_one<4, 8, 2, ARG>(a, pl, l, st, configure);
+    default: return cudaErrorInvalidConfiguration;
+    }
 }
 
 }  // namespace
@@ -465,7 +532,7 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     pl->tmb = pl->nms * 32 * pl->tm;
     pl->threads = (pl->nsg * pl->nms + 1) * 32;           // consumer warps + the producer warp
     // stages of ks * (tmb + sb) ints: aim at <= 40 KB each, 2..4 of them in the opt-in shared memory
-    const int avail = ctx->smem_optin - 2048;
+    const int avail = ctx->smem_optin - 2048 - kMaxStages * (2 * pl->sb + 4) * 4;
     const int row = (pl->tmb + pl->sb) * 4;
     int ks = (40 * 1024) / row;
     if (ks > S) ks = S;
@@ -478,7 +545,7 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     pl->nst = nst;
     pl->nkc = (S + ks - 1) / ks;
     pl->ntiles_m = (sh->M + 1 + pl->tmb - 1) / pl->tmb;
-    pl->smem = nst * ks * row;
+    pl->smem = nst * ks * row + nst * (2 * pl->sb + 4) * 4;
     const long long items = (long long)sh->B * pl->ntiles_m * pl->nsb;
     pl->grid = (int)(items < ctx->num_sms ? items : ctx->num_sms);
     return true;
@@ -486,11 +553,17 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
 
 cudaError_t galv_dp_configure(const galv_ctx* ctx)
 {
-    cudaError_t e;
-    e = cudaFuncSetAttribute(layer_tiled_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 2048);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(layer_tiled_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->smem_optin - 2048);
-    return e;
+    // opt every instantiation into the large dynamic shared memory once per context
+    DpArgs a{};
+    DpPlan pl{};
+    pl.smem = ctx->smem_optin - 2048;
+    for (int nsg = 1; nsg <= 8; ++nsg) {
+        pl.nsg = nsg;
+        cudaError_t e = launch_tiled<false>(a, pl, 0, nullptr, true);
+        if (e == cudaSuccess) e = launch_tiled<true>(a, pl, 0, nullptr, true);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a, cudaStream_t st)
@@ -530,7 +603,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
             layer_reference_kernel<<<dim3((unsigned)((size_t)B * mchunks), S, 1), 256, 0, st>>>(a, l);
             e = cudaGetLastError();
         } else {
-            e = a.A ? launch_tiled<4, true>(a, pl, l, st) : launch_tiled<4, false>(a, pl, l, st);
+            e = a.A ? launch_tiled<true>(a, pl, l, st, false) : launch_tiled<false>(a, pl, l, st, false);
         }
         if (e != cudaSuccess) return e;
     }
