@@ -191,12 +191,14 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 // consecutive items mostly share the instance (its trans rows stay in L2).  Warp roles:
 //   warp NC (producer): for every chunk (item, k-chunk of s') waits for a free stage, then
 //       bulk-copies KS rows of the previous layer's slice and the matching rows of trans into it;
-//       also writes the cells no column maps to (m < mem(l,s)) and the pad columns;
+//   warp NC+1 (helper): stages each item's record (mem and time row of the s-block, instance)
+//       next to the item's last chunk, and writes the cells no column maps to (m < mem(l,s))
+//       and the pad columns;
 //   warps 0..NC-1 (consumers): warp (ms, sg) keeps a TM x 8 register tile per lane
 //       (columns m' = tile + ms*32*TM + j*32 + lane, strategies sg*8 .. sg*8+7), waits for the
 //       stage, runs one fused add-min per relaxation, releases the stage, and after the last
 //       chunk stores column m' of strategy s at m' + mem(l,s).
-// Stages are handed over with mbarriers (full: bytes landed; empty: every consumer warp done),
+// Stages are handed over with mbarriers (full: bytes landed and record written; empty: every consumer warp done),
 // so there is no block-wide barrier in the loop.  Every wait is bounded.
 
 constexpr int kMaxStages = 4;
@@ -219,8 +221,20 @@ __device__ __forceinline__ void item_next(ItemPos& p, const DpPlan& pl) {
 // Shared memory: NST stages of [KS][TMB] previous-layer values + [KS][SB] trans values, then per
 // stage a small record the producer fills for the item whose last chunk sits in that stage:
 // mem(l,s) and time(l,s) of the s-block, the instance index and whether l is its last layer.
+// Items are dealt to CTAs by weight, not by count: a full tile weighs 64, the ragged last tile of
+// an instance (fewer than TMB columns) in proportion to its 32-column groups.  Returns the first
+// item whose cumulative weight reaches `target`.
+__device__ __forceinline__ long long item_at_weight(long long target, const DpPlan& pl, int wr) {
+    const long long full = (long long)(pl.ntiles_m - 1) * pl.nsb * 64;     // weight of an instance's full tiles
+    const long long per = full + (long long)pl.nsb * wr;
+    const long long oi = target / per;
+    const long long rem = target - oi * per;
+    const long long idx = rem < full ? (rem + 63) / 64 : (pl.ntiles_m - 1) * pl.nsb + (rem - full + wr - 1) / wr;
+    return oi * pl.ntiles_m * pl.nsb + idx;
+}
+
 template <int TM, int NSG, int NMS, bool ARG>
-__global__ void __launch_bounds__((NSG * NMS + 1) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l)
+__global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l)
 {
     constexpr int NC = NSG * NMS;                         // consumer warps
     constexpr int SB = NSG * TS;                          // strategies per item
@@ -235,8 +249,13 @@ __global__ void __launch_bounds__((NSG * NMS + 1) * 32, 1) layer_tiled_kernel(co
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
     const int KS = pl.ks, NKC = pl.nkc, NST = pl.nst;
 
-    const long long nitems = (long long)a.nactive[l] * pl.ntiles_m * pl.nsb;
-    const long long it0 = nitems * blockIdx.x / gridDim.x, it1 = nitems * (blockIdx.x + 1) / gridDim.x;
+    const int nact = a.nactive[l];
+    // weight of the last tile of an instance: its 32-column groups out of TMB/32, in 64ths
+    const int last_cols = M + 1 - (pl.ntiles_m - 1) * TMB;
+    const int wr = max(1, ((last_cols + 31) / 32) * 64 / (TMB / 32));
+    const long long wtot = (long long)nact * pl.nsb * ((long long)(pl.ntiles_m - 1) * 64 + wr);
+    const long long it0 = item_at_weight(wtot * blockIdx.x / gridDim.x, pl, wr);
+    const long long it1 = item_at_weight(wtot * (blockIdx.x + 1) / gridDim.x, pl, wr);
     if (it0 >= it1) return;
 
     int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
@@ -244,7 +263,7 @@ __global__ void __launch_bounds__((NSG * NMS + 1) * 32, 1) layer_tiled_kernel(co
     int32_t* const meta0 = stage0 + NST * stage_elems;
 
     if (tid == 0) {
-        for (int k = 0; k < NST; ++k) { mbar_init(&full_bar[k], 1); mbar_init(&empty_bar[k], NC); }
+        for (int k = 0; k < NST; ++k) { mbar_init(&full_bar[k], 2); mbar_init(&empty_bar[k], NC); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -262,8 +281,6 @@ __global__ void __launch_bounds__((NSG * NMS + 1) * 32, 1) layer_tiled_kernel(co
             const int w = min(TMB, m_pitch - m0);
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
-            const bool is_last = (a.L[i] == l + 1);
-            const size_t qrow = ((size_t)i * a.Lmax + l) * S;
             const int32_t* prev = (a.C ? a.C + ((size_t)i * a.Lmax + (l - 1)) * slice
                                        : a.roll + ((size_t)((l - 1) & 1) * a.B + i) * slice) + m0;
             const int32_t* T = a.trans_q + (size_t)i * S * S + sb0;
@@ -283,16 +300,8 @@ __global__ void __launch_bounds__((NSG * NMS + 1) * 32, 1) layer_tiled_kernel(co
                         const int r = e / sbw, c = e - r * sbw;
                         ts[r * SB + c] = __ldg(T + (size_t)(k0 + r) * S + c);
                     }
+                    __syncwarp();
                 }
-                if (kc == NKC - 1) {
-                    int32_t* meta = meta0 + st * META;
-                    for (int c = lane; c < sbw; c += 32) {
-                        meta[c] = __ldg(a.mem_q + qrow + sb0 + c);
-                        meta[SB + c] = __ldg(a.time_q + qrow + sb0 + c);
-                    }
-                    if (lane == 0) { meta[2 * SB] = i; meta[2 * SB + 1] = is_last; }
-                }
-                __syncwarp();
                 if (lane == 0)
                     mbar_expect_tx(&full_bar[st], (uint32_t)kn * (uint32_t)(w + (bulk_t ? sbw : 0)) * 4u);
                 __syncwarp();
@@ -301,14 +310,47 @@ __global__ void __launch_bounds__((NSG * NMS + 1) * 32, 1) layer_tiled_kernel(co
                     if (bulk_t) bulk_g2s(ts + r * SB, T + (size_t)(k0 + r) * S, (uint32_t)sbw * 4u, &full_bar[st]);
                 }
             }
+        }
+        return;
+    }
+    if (warp == NC + 1) {
+        // ------------------------------------------------------------ helper
+        int n = 0;
+        for (long long item = it0; item < it1; ++item, item_next(pos, pl)) {
+            const int i = a.order[pos.oi];
+            const int sb0 = pos.sb * SB;
+            const int sbw = min(SB, S - sb0);
+            const int is_last = (a.L[i] == l + 1);
+            const size_t qrow = ((size_t)i * a.Lmax + l) * S + sb0;
+            // this s-block's mem and time row, two strategies per lane (SB <= 64)
+            const int mq0 = lane < sbw ? __ldg(a.mem_q + qrow + lane) : 0;
+            const int mq1 = lane + 32 < sbw ? __ldg(a.mem_q + qrow + lane + 32) : 0;
+            const int tq0 = lane < sbw ? __ldg(a.time_q + qrow + lane) : 0;
+            const int tq1 = lane + 32 < sbw ? __ldg(a.time_q + qrow + lane + 32) : 0;
+            for (int kc = 0; kc < NKC; ++kc, ++n) {
+                const int st = n % NST;
+                if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+                if (kc == NKC - 1) {
+                    int32_t* meta = meta0 + st * META;
+                    if (lane < SB) { meta[lane] = mq0; meta[SB + lane] = tq0; }
+                    if (lane + 32 < SB) { meta[lane + 32] = mq1; meta[SB + lane + 32] = tq1; }
+                    if (lane == 0) { meta[2 * SB] = i; meta[2 * SB + 1] = is_last; }
+                    __syncwarp();
+                }
+                if (lane == 0) mbar_arrive(&full_bar[st]);
+            }
             if (pos.mt == 0) {
                 // Cells no column maps to: m < mem(l,s), and the pad columns.
                 int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
                 int32_t* last = a.C_last + (size_t)i * slice;
                 uint8_t* aout = ARG ? a.A + ((size_t)i * a.Lmax + l) * slice : nullptr;
-                for (int s = sb0; s < sb0 + sbw; ++s) {
-                    const int lo = min(__ldg(a.mem_q + qrow + s), M + 1);
-                    const size_t o = (size_t)s * m_pitch;
+                for (int c = 0; c < sbw; ++c) {
+                    const int mq = __shfl_sync(0xffffffffu, c < 32 ? mq0 : mq1, c & 31);
+                    const int lo = min(mq, M + 1);
+                    const size_t o = (size_t)(sb0 + c) * m_pitch;
                     for (int m = lane; m < lo + (m_pitch - M - 1); m += 32) {
                         const int mm = m < lo ? m : m - lo + M + 1;
                         out[o + mm] = kInf;
@@ -320,7 +362,6 @@ __global__ void __launch_bounds__((NSG * NMS + 1) * 32, 1) layer_tiled_kernel(co
         }
         return;
     }
-    if (warp > NC) return;
 
     // ---------------------------------------------------------------- consumers
     const int sg = warp % NSG, ms = warp / NSG;
@@ -478,7 +519,7 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st
 {
     auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG>;
     if (configure) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
-    kern<<<pl.grid, (NSG * NMS + 1) * 32, pl.smem, st>>>(a, pl, l);
+    kern<<<pl.grid, (NSG * NMS + 2) * 32, pl.smem, st>>>(a, pl, l);
     return cudaGetLastError();
 }
 
@@ -530,7 +571,7 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     pl->nms = 16 / pl->nsg;
     if (pl->nms < 1) pl->nms = 1;
     pl->tmb = pl->nms * 32 * pl->tm;
-    pl->threads = (pl->nsg * pl->nms + 1) * 32;           // consumer warps + the producer warp
+    pl->threads = (pl->nsg * pl->nms + 2) * 32;           // consumer warps + producer + helper
     // stages of ks * (tmb + sb) ints: aim at <= 40 KB each, 2..4 of them in the opt-in shared memory
     const int avail = ctx->smem_optin - 2048 - kMaxStages * (2 * pl->sb + 4) * 4;
     const int row = (pl->tmb + pl->sb) * 4;

@@ -29,7 +29,7 @@ struct DpPlan {
     int nkc;       // chunks per item = ceil(S / ks)
     int nst;       // pipeline stages in shared memory
     int ntiles_m;  // ceil((M+1) / tmb)
-    int threads;   // (nsg * nms + 1) * 32: consumer warps and one producer warp
+    int threads;   // (nsg * nms + 2) * 32: consumer warps, producer warp, helper warp
     int smem;      // dynamic shared memory bytes
     int grid;      // resident CTAs
 };
