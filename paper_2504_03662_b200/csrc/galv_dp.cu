@@ -17,6 +17,10 @@
 // One launch per layer (a layer needs all of the previous one); launches are
 // plain stream work, so a caller may capture the whole search in a CUDA graph.
 
+#include <cuda.h>
+
+#include <cstring>
+
 #include "galv_internal.h"
 
 namespace {
@@ -35,6 +39,13 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// 2-D tiled TMA load: the box at element coordinates (x, y) of the tensor behind `map` lands densely
+// (row-major, box rows of box-width elements) at dst; the box's full byte count is signalled on bar,
+// out-of-range elements are filled with zeros.  x * 4 bytes must be a multiple of 16.
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -234,12 +245,17 @@ __device__ __forceinline__ long long item_at_weight(long long target, const DpPl
 }
 
 template <int TM, int NSG, int NMS, bool ARG>
-__global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l)
+__global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l,
+                                                                              const __grid_constant__ CUtensorMap map_c,
+                                                                              const __grid_constant__ CUtensorMap map_t)
 {
     constexpr int NC = NSG * NMS;                         // consumer warps
     constexpr int SB = NSG * TS;                          // strategies per item
     constexpr int TMB = NMS * 32 * TM;                    // columns per item
+    constexpr int BOXC = 32 * TM * ((NMS % 2 == 0 && 64 * TM <= 256) ? 2 : 1);   // columns per TMA box (box extents are <= 256)
+    constexpr int NBOX = TMB / BOXC;
     constexpr int META = 2 * SB + 4;
+    static_assert(TMB % BOXC == 0 && BOXC % (32 * TM) == 0, "a warp's columns must sit inside one box");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
@@ -258,8 +274,9 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
     const long long it1 = item_at_weight(wtot * (blockIdx.x + 1) / gridDim.x, pl, wr);
     if (it0 >= it1) return;
 
+    // stage: NBOX boxes of [KS][BOXC] previous-layer values, then [KS][SB] trans values; 128-byte multiples
     int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
-    const int stage_elems = KS * (TMB + SB);
+    const int stage_elems = (KS * (TMB + SB) + 31) & ~31;
     int32_t* const meta0 = stage0 + NST * stage_elems;
 
     if (tid == 0) {
@@ -273,16 +290,16 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
 
     if (warp == NC) {
         // ------------------------------------------------------------ producer
-        const bool bulk_t = (S & 3) == 0;                 // trans rows 16-byte aligned
+        const bool tma_t = pl.tma_t != 0;                 // trans rows 16-byte aligned: one box per chunk
+        const int row0 = a.C ? (l - 1) * S : ((l - 1) & 1) * a.B * S;      // row of (instance 0, layer l-1, s'=0)
+        const int inst_rows = a.C ? a.Lmax * S : S;
         int n = 0;                                        // chunk counter
         for (long long item = it0; item < it1; ++item, item_next(pos, pl)) {
             const int i = a.order[pos.oi];
             const int m0 = pos.mt * TMB;
-            const int w = min(TMB, m_pitch - m0);
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
-            const int32_t* prev = (a.C ? a.C + ((size_t)i * a.Lmax + (l - 1)) * slice
-                                       : a.roll + ((size_t)((l - 1) & 1) * a.B + i) * slice) + m0;
+            const int yc = row0 + i * inst_rows;
             const int32_t* T = a.trans_q + (size_t)i * S * S + sb0;
             for (int kc = 0; kc < NKC; ++kc, ++n) {
                 const int st = n % NST;
@@ -291,24 +308,26 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
                     return;
                 }
                 const int k0 = kc * KS;
-                const int kn = min(KS, S - k0);
                 int32_t* cs = stage0 + st * stage_elems;
                 int32_t* ts = cs + KS * TMB;
-                if (!bulk_t) {
+                if (!tma_t) {
                     // unaligned trans rows: plain copies by this warp, published by the arrive below
+                    const int kn = min(KS, S - k0);
                     for (int e = lane; e < kn * sbw; e += 32) {
                         const int r = e / sbw, c = e - r * sbw;
                         ts[r * SB + c] = __ldg(T + (size_t)(k0 + r) * S + c);
                     }
                     __syncwarp();
                 }
-                if (lane == 0)
-                    mbar_expect_tx(&full_bar[st], (uint32_t)kn * (uint32_t)(w + (bulk_t ? sbw : 0)) * 4u);
-                __syncwarp();
-                for (int r = lane; r < kn; r += 32) {
-                    bulk_g2s(cs + r * TMB, prev + (size_t)(k0 + r) * m_pitch, (uint32_t)w * 4u, &full_bar[st]);
-                    if (bulk_t) bulk_g2s(ts + r * SB, T + (size_t)(k0 + r) * S, (uint32_t)sbw * 4u, &full_bar[st]);
+                if (lane == 0) {
+                    // boxes always deliver their full size (zeros beyond the tensor's edge)
+                    mbar_expect_tx(&full_bar[st], (uint32_t)KS * (uint32_t)(TMB + (tma_t ? SB : 0)) * 4u);
+#pragma unroll
+                    for (int bx = 0; bx < NBOX; ++bx)
+                        tma_load_2d(cs + bx * KS * BOXC, &map_c, m0 + bx * BOXC, yc + k0, &full_bar[st]);
+                    if (tma_t) tma_load_2d(ts, &map_t, sb0, i * S + k0, &full_bar[st]);
                 }
+                __syncwarp();
             }
         }
         return;
@@ -389,7 +408,8 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
             }
             const int k0 = kc * KS;
             const int kn = min(KS, S - k0);
-            const int32_t* cs = stage0 + st * stage_elems + ms * (32 * TM) + lane;
+            // this warp's columns inside their box, and its 8 trans columns
+            const int32_t* cs = stage0 + st * stage_elems + ((ms * (32 * TM)) / BOXC) * (KS * BOXC) + (ms * (32 * TM)) % BOXC + lane;
             const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
             if (nj == TM) {
                 int k = 0;
@@ -398,7 +418,7 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
                     for (int kk = 0; kk < 4; ++kk) {
                         int c[TM];
 #pragma unroll
-                        for (int j = 0; j < TM; ++j) c[j] = cs[kk * TMB + j * 32];
+                        for (int j = 0; j < TM; ++j) c[j] = cs[kk * BOXC + j * 32];
                         const int4 t0 = *reinterpret_cast<const int4*>(ts + kk * SB);
                         const int4 t1 = *reinterpret_cast<const int4*>(ts + kk * SB + 4);
                         const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
@@ -414,7 +434,7 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
                                 }
                             }
                     }
-                    cs += 4 * TMB;
+                    cs += 4 * BOXC;
                     ts += 4 * SB;
                 }
                 for (; k < kn; ++k) {
@@ -430,7 +450,7 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
                             if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
                         }
                     }
-                    cs += TMB;
+                    cs += BOXC;
                     ts += SB;
                 }
             } else if (nj > 0) {
@@ -442,7 +462,7 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
 #pragma unroll
                     for (int j = 0; j < TM; ++j)
                         if (j < nj) {
-                            const int c = cs[k * TMB + j * 32];
+                            const int c = cs[k * BOXC + j * 32];
 #pragma unroll
                             for (int u = 0; u < TS; ++u) {
                                 const int cand = c + t[u];
@@ -515,27 +535,27 @@ __global__ void finalize_kernel(int B, const int32_t* err, int32_t* status)
 }
 
 template <int TM, int NSG, int NMS, bool ARG>
-cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st, bool configure)
+cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st, const CUtensorMap* maps)
 {
     auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG>;
-    if (configure) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
-    kern<<<pl.grid, (NSG * NMS + 2) * 32, pl.smem, st>>>(a, pl, l);
+    if (!maps) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+    kern<<<pl.grid, (NSG * NMS + 2) * 32, pl.smem, st>>>(a, pl, l, maps[0], maps[1]);
     return cudaGetLastError();
 }
 
 // nsg warps along s, 16/nsg (rounded down) along m: one instantiation per s-block width.
 template <bool ARG>
-cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st, bool configure)
+cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st, const CUtensorMap* maps)
 {
     switch (pl.nsg) {
-    case 1: return launch_one<4, 1, 16, ARG>(a, pl, l, st, configure);
-    case 2: return launch_one<4, 2, 8, ARG>(a, pl, l, st, configure);
-    case 3: return launch_one<4, 3, 5, ARG>(a, pl, l, st, configure);
-    case 4: return launch_one<4, 4, 4, ARG>(a, pl, l, st, configure);
-    case 5: return launch_one<4, 5, 3, ARG>(a, pl, l, st, configure);
-    case 6: return launch_one<4, 6, 2, ARG>(a, pl, l, st, configure);
-    case 7: return launch_one<4, 7, 2, ARG>(a, pl, l, st, configure);
-    case 8: return launch_one<4, 8, 2, ARG>(a, pl, l, st, configure);
+    case 1: return launch_one<4, 1, 16, ARG>(a, pl, l, st, maps);
+    case 2: return launch_one<4, 2, 8, ARG>(a, pl, l, st, maps);
+    case 3: return launch_one<4, 3, 5, ARG>(a, pl, l, st, maps);
+    case 4: return launch_one<4, 4, 4, ARG>(a, pl, l, st, maps);
+    case 5: return launch_one<4, 5, 3, ARG>(a, pl, l, st, maps);
+    case 6: return launch_one<4, 6, 2, ARG>(a, pl, l, st, maps);
+    case 7: return launch_one<4, 7, 2, ARG>(a, pl, l, st, maps);
+    case 8: return launch_one<4, 8, 2, ARG>(a, pl, l, st, maps);
     default: return cudaErrorInvalidConfiguration;
     }
 }
@@ -545,6 +565,10 @@ cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t 
 // ---------------------------------------------------------------- host side
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 WsLayout galv_ws_layout(const galv_shape* sh)
 {
@@ -579,17 +603,40 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     if (ks > S) ks = S;
     if (ks >= 8) ks &= ~7;
     if (ks < 1) ks = 1;
-    int nst = avail / (ks * row);
+    const int stage_bytes = (ks * row + 127) & ~127;
+    int nst = avail / stage_bytes;
     if (nst > kMaxStages) nst = kMaxStages;
     if (nst < 2) return false;
     pl->ks = ks;
     pl->nst = nst;
     pl->nkc = (S + ks - 1) / ks;
     pl->ntiles_m = (sh->M + 1 + pl->tmb - 1) / pl->tmb;
-    pl->smem = nst * ks * row + nst * (2 * pl->sb + 4) * 4;
+    pl->smem = nst * stage_bytes + nst * (2 * pl->sb + 4) * 4;
+    pl->tma_t = (S % 4) == 0;                             // trans row pitch a multiple of 16 bytes
     const long long items = (long long)sh->B * pl->ntiles_m * pl->nsb;
     pl->grid = (int)(items < ctx->num_sms ? items : ctx->num_sms);
     return true;
+}
+
+// Tensor map of a row-major int32 matrix [rows][cols] (row pitch = cols * 4 bytes) with a dense box.
+static cudaError_t encode_2d(CUtensorMap* map, void* base, size_t cols, size_t rows, int box_cols, int box_rows)
+{
+    static PFN_encodeTiled fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+        if (e != cudaSuccess) return e;
+        if (q != cudaDriverEntryPointSuccess || !p) return cudaErrorNotSupported;
+        fn = reinterpret_cast<PFN_encodeTiled>(p);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_INT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
 cudaError_t galv_dp_configure(const galv_ctx* ctx)
@@ -600,8 +647,8 @@ cudaError_t galv_dp_configure(const galv_ctx* ctx)
     pl.smem = ctx->smem_optin - 2048;
     for (int nsg = 1; nsg <= 8; ++nsg) {
         pl.nsg = nsg;
-        cudaError_t e = launch_tiled<false>(a, pl, 0, nullptr, true);
-        if (e == cudaSuccess) e = launch_tiled<true>(a, pl, 0, nullptr, true);
+        cudaError_t e = launch_tiled<false>(a, pl, 0, nullptr, nullptr);
+        if (e == cudaSuccess) e = launch_tiled<true>(a, pl, 0, nullptr, nullptr);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -637,6 +684,16 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     const bool reference = (sh->flags & GALV_KERNEL_REFERENCE) != 0;
     DpPlan pl;
     if (!reference && !galv_dp_make_plan(ctx, sh, &pl)) return cudaErrorInvalidConfiguration;
+    CUtensorMap maps[2];
+    std::memset(maps, 0, sizeof(maps));
+    if (!reference) {
+        // previous-layer values as a 2-D tensor [rows of m_pitch columns]; box = ks rows x (<=256) columns
+        const int boxc = 32 * pl.tm * ((pl.nms % 2 == 0 && 64 * pl.tm <= 256) ? 2 : 1);
+        const size_t rows = a.C ? (size_t)B * Lmax * S : (size_t)2 * B * S;
+        if ((e = encode_2d(&maps[0], a.C ? (void*)a.C : (void*)a.roll, (size_t)a.m_pitch, rows, boxc, pl.ks)) != cudaSuccess) return e;
+        if (pl.tma_t &&
+            (e = encode_2d(&maps[1], (void*)a.trans_q, (size_t)S, (size_t)B * S, pl.sb, pl.ks)) != cudaSuccess) return e;
+    }
     if (ctx->profiling) cudaEventRecord(ctx->ev0, st);
     for (int l = 1; l < Lmax; ++l) {
         if (reference) {
@@ -644,7 +701,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
             layer_reference_kernel<<<dim3((unsigned)((size_t)B * mchunks), S, 1), 256, 0, st>>>(a, l);
             e = cudaGetLastError();
         } else {
-            e = a.A ? launch_tiled<true>(a, pl, l, st, false) : launch_tiled<false>(a, pl, l, st, false);
+            e = a.A ? launch_tiled<true>(a, pl, l, st, maps) : launch_tiled<false>(a, pl, l, st, maps);
         }
         if (e != cudaSuccess) return e;
     }

@@ -28,6 +28,7 @@ struct DpPlan {
     int ks;        // previous-layer strategies staged per pipeline stage
     int nkc;       // chunks per item = ceil(S / ks)
     int nst;       // pipeline stages in shared memory
+    int tma_t;     // trans rows are 16-byte aligned: staged by a tiled TMA box, else by plain copies
     int ntiles_m;  // ceil((M+1) / tmb)
     int threads;   // (nsg * nms + 2) * 32: consumer warps, producer warp, helper warp
     int smem;      // dynamic shared memory bytes
