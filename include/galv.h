@@ -145,6 +145,35 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
                    int32_t* status, void* stream);
 
 /*
+ * The same search without any caller-provided scratch (the paper has no
+ * counterpart; this exists for deployment).  Some callers cannot call
+ * cudaMalloc at all: a plugin running inside a host application that owns the
+ * device heap, code on a latency path where an allocation (which may
+ * synchronise the device) is forbidden, or a process whose memory pool was
+ * sized up front and is full.  For them the scratch that galv_dp_search takes
+ * as `workspace` lives in a fixed array of GALV_STATIC_WORKSPACE_BYTES inside
+ * the library's device image; every GPU that loads the library carries that
+ * array until the process exits.  Inputs and outputs are still the caller's.
+ *
+ * Arguments, results and status bits are those of galv_dp_search.  Shapes whose
+ * galv_dp_workspace_bytes exceeds GALV_STATIC_WORKSPACE_BYTES are refused with
+ * GALV_ERR_WORKSPACE (in practice: any batch that keeps the full table fits;
+ * the rolling two-layer mode fits only small B*S*m_pitch).  The call itself
+ * allocates nothing, on the host or the device.
+ *
+ * The first call on a device looks up the array's device address (once per
+ * device); make that first call outside any stream capture.  All calls share
+ * the one array: what has to start from zero is cleared by each call, and two
+ * calls that overlap on the GPU (different streams, or different contexts on
+ * the same device) race on it — serialise them.
+ */
+#define GALV_STATIC_WORKSPACE_BYTES (1 << 20)
+int galv_dp_search_static(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                          const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,
+                          int32_t* C, uint8_t* A, int32_t* C_last,
+                          int32_t* status, void* stream);
+
+/*
  * Optimum and plan (Section 3: the selector's output is a per-layer
  * parallelism plan).  For every instance, at budget[i] (NULL: M):
  *   opt_cost = min_s C_last[budget][s], lowest s on ties (GALV_INF if none is finite);

@@ -17,12 +17,13 @@ INF = 2 ** 30 - 1
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 STATUS_INFEASIBLE, STATUS_BAD_INPUT, STATUS_OVERFLOW_RISK, STATUS_TIMEOUT = 1, 2, 4, 8
 STORE_C_FULL, STORE_ARGMIN, KERNEL_REFERENCE = 1, 2, 256
+STATIC_WORKSPACE_BYTES = 1 << 20
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgalv.so")
 
 EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "galv_eval_costs",
            "galv_dp_workspace_bytes", "galv_dp_search", "galv_backtrack", "galv_search_host_arena_bytes",
-           "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms")
+           "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_dp_search_static")
 
 
 class galv_shape(C.Structure):
@@ -60,6 +61,7 @@ def load_library() -> C.CDLL:
     lib.galv_dp_workspace_bytes.restype = sz
     lib.galv_dp_search.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.galv_backtrack.argtypes = [vp, shp] + [vp] * 13
+    lib.galv_dp_search_static.argtypes = [vp, shp] + [vp] * 9
     lib.galv_search_host_arena_bytes.argtypes = [vp, shp, C.c_int]
     lib.galv_search_host_arena_bytes.restype = sz
     lib.galv_search_host.argtypes = [vp, shp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -126,6 +128,12 @@ class Galv:
                                             _ptr(Ct), _ptr(At), _ptr(C_last), _ptr(workspace),
                                             0 if workspace is None else workspace.numel() * workspace.element_size(),
                                             _ptr(status), _stream()))
+
+    def galv_dp_search_static(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, status):
+        """galv_dp_search on the library's built-in scratch array: nothing is allocated, the caller passes no workspace."""
+        self._check(self.lib.galv_dp_search_static(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q),
+                                                   _ptr(trans_q), _ptr(Ct), _ptr(At), _ptr(C_last), _ptr(status),
+                                                   _stream()))
 
     def galv_backtrack(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, budget, opt_cost, plan, mem_used, status):
         self._check(self.lib.galv_backtrack(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),

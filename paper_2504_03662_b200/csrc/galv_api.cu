@@ -61,6 +61,12 @@ Arena arena_layout(const galv_shape* sh, bool with_model)
 
 }  // namespace
 
+int galv_set_error(galv_ctx* ctx, int code, const char* text)
+{
+    if (ctx) std::snprintf(ctx->err, sizeof(ctx->err), "%s", text);
+    return code;
+}
+
 extern "C" {
 
 int galv_create(galv_ctx** out, int device_ordinal)

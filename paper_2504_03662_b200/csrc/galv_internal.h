@@ -52,6 +52,9 @@ struct DpArgs {
     int32_t* status;
 };
 
+// records `text` as the context's last error and returns `code`
+int galv_set_error(galv_ctx* ctx, int code, const char* text);
+
 // workspace carve-up (offsets in bytes, all 256-aligned)
 struct WsLayout { size_t order, nactive, scratch, err, roll, total; };
 WsLayout galv_ws_layout(const galv_shape* sh);
