@@ -37,6 +37,9 @@ METRIC, UNIT = "dp_cell_updates_per_s", "cells/s"
 # Integer-ALU peak of one B200: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min
 # (one min-plus relaxation) per lane per clock.
 ALU_PEAK_GOPS = 148 * 64 * 1.965
+# DRAM bytes (read + write) of one layer_tiled_kernel launch, from the committed ncu captures under
+# profiles/ (a capture launch covers the same units as a benchmark launch: every instance, one layer).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"config3_heterogeneous": 498.0e6, "config4_research_sweep": 509.2e6}
 
 
 def workload_for(k: int, rank: int = 0, batch: int = 0, layers: int = 0):
@@ -281,7 +284,9 @@ def main():
         "searches_per_s": world * w.B * args.steps / t, "relaxations_per_s": world * w.relaxations * args.steps / t,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(w) * args.steps,
         "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_GOPS, "unit": "G add-min/s",
-                     "frac": achieved / ALU_PEAK_GOPS, "traffic": None,
+                     "frac": achieved / ALU_PEAK_GOPS, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
+                     "traffic_unit": "bytes per launch (ncu dram read+write)",
+                     "algorithmic_bytes_per_launch": 2 * 4 * w.B * w.S * w.m_pitch,
                      "kernel": "layer_tiled_kernel", "launch_ms": r["layer_kernel_ms_avg"],
                      "peak_source": "derived: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min per lane per clock"},
     }
