@@ -47,6 +47,13 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// 1-D bulk async store shared -> global (both 16-byte aligned, bytes a multiple of 16), tracked in bulk groups.
+__device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(src)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -153,12 +160,10 @@ __global__ void base_layer_kernel(DpArgs a)
     const int mm = a.mem_q[(size_t)i * a.Lmax * a.S + s];
     const size_t row = ((size_t)i * a.S + s) * a.m_pitch;
     int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax * a.S + s) * a.m_pitch : a.roll + row;
-    int32_t* last = (a.L[i] == 1) ? a.C_last + row : nullptr;
     uint8_t* ao = a.A ? a.A + ((size_t)i * a.Lmax * a.S + s) * a.m_pitch : nullptr;
     for (int m = blockIdx.x * blockDim.x + threadIdx.x; m < a.m_pitch; m += gridDim.x * blockDim.x) {
         const int v = (m <= a.M && mm <= m) ? tt : kInf;
         out[m] = v;
-        if (last) last[m] = v;
         if (ao) ao[m] = 255;
     }
 }
@@ -192,7 +197,6 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
     }
     const int v = best < kInf ? best + tt : kInf;
     out[(size_t)s * a.m_pitch + m] = v;
-    if (a.L[i] == l + 1) a.C_last[((size_t)i * a.S + s) * a.m_pitch + m] = v;
     if (a.A) a.A[(((size_t)i * a.Lmax + l) * a.S + s) * a.m_pitch + m] = (uint8_t)arg;
 }
 
@@ -205,10 +209,16 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 //   warp NC+1 (helper): stages each item's record (mem and time row of the s-block, instance)
 //       next to the item's last chunk, and writes the cells no column maps to (m < mem(l,s))
 //       and the pad columns;
+//   warp NC+2 (store warp): sends the finished item's outputs from a staging tile in shared memory
+//       to the table, one bulk async store (TMA) per row, while the consumers already work on the
+//       next item.  The SM's store port takes 32 bytes per clock whoever feeds it; fed by plain
+//       stores of the consumers it also holds up their shared-memory loads, the TMA unit reads
+//       shared memory on its own path;
 //   warps 0..NC-1 (consumers): warp (ms, sg) keeps a TM x 8 register tile per lane
 //       (columns m' = tile + ms*32*TM + j*32 + lane, strategies sg*8 .. sg*8+7), waits for the
 //       stage, runs one fused add-min per relaxation, releases the stage, and after the last
-//       chunk stores column m' of strategy s at m' + mem(l,s).
+//       chunk adds time(l,s) and writes its tile into the staging tile, row s shifted by
+//       mem(l,s) mod 4 so that column m' + mem(l,s) of the table is 16-byte aligned with it.
 // Stages are handed over with mbarriers (full: bytes landed and record written; empty: every consumer warp done),
 // so there is no block-wide barrier in the loop.  Every wait is bounded.
 
@@ -231,7 +241,8 @@ __device__ __forceinline__ void item_next(ItemPos& p, const DpPlan& pl) {
 
 // Shared memory: NST stages of [KS][TMB] previous-layer values + [KS][SB] trans values, then per
 // stage a small record the producer fills for the item whose last chunk sits in that stage:
-// mem(l,s) and time(l,s) of the s-block, the instance index and whether l is its last layer.
+// mem(l,s) and time(l,s) of the s-block and the instance index; then the staging tile of the
+// outputs and its header.
 // Items are dealt to CTAs by weight, not by count: a full tile weighs 64, the ragged last tile of
 // an instance (fewer than TMB columns) in proportion to its 32-column groups.  Returns the first
 // item whose cumulative weight reaches `target`.
@@ -245,7 +256,7 @@ __device__ __forceinline__ long long item_at_weight(long long target, const DpPl
 }
 
 template <int TM, int NSG, int NMS, bool ARG>
-__global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l,
+__global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l,
                                                                               const __grid_constant__ CUtensorMap map_c,
                                                                               const __grid_constant__ CUtensorMap map_t)
 {
@@ -255,11 +266,13 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
     constexpr int BOXC = 32 * TM * ((NMS % 2 == 0 && 64 * TM <= 256) ? 2 : 1);   // columns per TMA box (box extents are <= 256)
     constexpr int NBOX = TMB / BOXC;
     constexpr int META = 2 * SB + 4;
+    constexpr int RS = TMB + 4;                           // staging row: TMB columns + room for the shift
     static_assert(TMB % BOXC == 0 && BOXC % (32 * TM) == 0, "a warp's columns must sit inside one box");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t out_full, out_empty;  // staging tile written / drained
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
@@ -278,9 +291,14 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
     int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
     const int stage_elems = (KS * (TMB + SB) + 31) & ~31;
     int32_t* const meta0 = stage0 + NST * stage_elems;
+    // staging tile [SB][RS] + its header: mem(l,s) per row, instance, last-layer flag
+    int32_t* const stg0 = meta0 + ((NST * META + 31) & ~31);
+    int32_t* const hdr0 = stg0 + SB * RS;
 
     if (tid == 0) {
         for (int k = 0; k < NST; ++k) { mbar_init(&full_bar[k], 2); mbar_init(&empty_bar[k], NC); }
+        mbar_init(&out_full, NC);
+        mbar_init(&out_empty, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -339,7 +357,6 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
             const int i = a.order[pos.oi];
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);
-            const int is_last = (a.L[i] == l + 1);
             const size_t qrow = ((size_t)i * a.Lmax + l) * S + sb0;
             // this s-block's mem and time row, two strategies per lane (SB <= 64)
             const int mq0 = lane < sbw ? __ldg(a.mem_q + qrow + lane) : 0;
@@ -356,7 +373,7 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
                     int32_t* meta = meta0 + st * META;
                     if (lane < SB) { meta[lane] = mq0; meta[SB + lane] = tq0; }
                     if (lane + 32 < SB) { meta[lane + 32] = mq1; meta[SB + lane + 32] = tq1; }
-                    if (lane == 0) { meta[2 * SB] = i; meta[2 * SB + 1] = is_last; }
+                    if (lane == 0) meta[2 * SB] = i;
                     __syncwarp();
                 }
                 if (lane == 0) mbar_arrive(&full_bar[st]);
@@ -364,7 +381,6 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
             if (pos.mt == 0) {
                 // Cells no column maps to: m < mem(l,s), and the pad columns.
                 int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
-                int32_t* last = a.C_last + (size_t)i * slice;
                 uint8_t* aout = ARG ? a.A + ((size_t)i * a.Lmax + l) * slice : nullptr;
                 for (int c = 0; c < sbw; ++c) {
                     const int mq = __shfl_sync(0xffffffffu, c < 32 ? mq0 : mq1, c & 31);
@@ -373,12 +389,51 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
                     for (int m = lane; m < lo + (m_pitch - M - 1); m += 32) {
                         const int mm = m < lo ? m : m - lo + M + 1;
                         out[o + mm] = kInf;
-                        if (is_last) last[o + mm] = kInf;
                         if (ARG) aout[o + mm] = 255;
                     }
                 }
             }
         }
+        return;
+    }
+
+    if (warp == NC + 2) {
+        // ------------------------------------------------------------ store warp
+        // Staging row `row` holds strategy sb0+row shifted by r = mem mod 4: staging column x is table
+        // column g0 + x with g0 = m0 + mem - r a multiple of 4.  Columns r .. r+TMB-1 are real, and
+        // table columns above M do not exist.  Each lane takes rows lane, lane+32: the 16-byte aligned
+        // middle leaves as one bulk store, the few cells before and after it as plain stores.
+        int it = 0;
+        for (long long item = it0; item < it1; ++item, item_next(pos, pl), ++it) {
+            if (!mbar_wait(&out_full, it & 1)) {
+                if (lane == 0) atomicExch(a.err, 1);
+                return;
+            }
+            const int i = hdr0[SB];
+            const int m0 = pos.mt * TMB;
+            const int sb0 = pos.sb * SB;
+            const int sbw = min(SB, S - sb0);
+            int32_t* out = (a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice)
+                           + (size_t)sb0 * m_pitch;
+            for (int row = lane; row < sbw; row += 32) {
+                const int mm = hdr0[row];
+                const int r = mm & 3;
+                const int g0 = m0 + mm - r;
+                const int hi = min(r + TMB, M + 1 - g0);          // first staging column not to store
+                if (hi <= r) continue;
+                const int32_t* src = stg0 + row * RS;
+                int32_t* dst = out + (size_t)row * m_pitch + (size_t)g0;
+                const int lo4 = r ? 4 : 0, hi4 = hi & ~3;         // aligned middle [lo4, hi4)
+                if (hi4 > lo4) bulk_s2g(dst + lo4, src + lo4, (uint32_t)(hi4 - lo4) * 4u);
+                for (int x = r; x < min(lo4, hi); ++x) dst[x] = src[x];
+                for (int x = max(hi4, lo4); x < hi; ++x) dst[x] = src[x];
+            }
+            bulk_commit();
+            bulk_wait_read();                                     // the staging tile may be overwritten
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&out_empty);
+        }
+        bulk_wait_all();
         return;
     }
 
@@ -399,7 +454,7 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
                 acc[j][u] = kInf;                            // min over candidates never exceeds kInf
                 if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = 255;
             }
-        int mm[TS], tt[TS], inst = 0, is_last = 0;
+        int mm[TS], tt[TS], inst = 0;
         for (int kc = 0; kc < NKC; ++kc, ++n) {
             const int st = n % NST;
             if (!mbar_wait(&full_bar[st], (n / NST) & 1)) {
@@ -481,49 +536,67 @@ __global__ void __launch_bounds__((NSG * NMS + 2) * 32, 1) layer_tiled_kernel(co
                 mm[0] = m0v.x; mm[1] = m0v.y; mm[2] = m0v.z; mm[3] = m0v.w; mm[4] = m1v.x; mm[5] = m1v.y; mm[6] = m1v.z; mm[7] = m1v.w;
                 tt[0] = t0v.x; tt[1] = t0v.y; tt[2] = t0v.z; tt[3] = t0v.w; tt[4] = t1v.x; tt[5] = t1v.y; tt[6] = t1v.z; tt[7] = t1v.w;
                 inst = meta[2 * SB];
-                is_last = meta[2 * SB + 1];
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);      // this warp is done reading the stage
         }
 
-        // Epilogue: column m' of strategy s lands at m = m' + mem(l,s).
-        if (nj > 0) {
-            const int i = inst;
-            int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
-            const int s0 = pos.sb * SB + sg * TS;
-            const int base = M - mw - lane;                  // group j of strategy u is stored iff j*32 + mem <= base
+        // Epilogue: add time(l,s) and hand the tile to the store warps through the staging tile;
+        // row s is written shifted by mem(l,s) mod 4 (see the store warps).
+        const int it = (int)(item - it0);
+        if (it > 0 && !mbar_wait(&out_empty, (it - 1) & 1)) {    // the previous item has been drained
+            if (lane == 0) atomicExch(a.err, 1);
+            return;
+        }
+        {
+            const int s0l = sg * TS;                          // first strategy of this warp inside the block
+            const int col = ms * (32 * TM) + lane;
 #pragma unroll
             for (int u = 0; u < TS; ++u) {
-                if (s0 + u < S) {
-                    const int lim = base - mm[u];
-                    const size_t o = (size_t)(s0 + u) * m_pitch + (size_t)(mm[u] + mw + lane);
-                    int32_t* po = out + o;
-                    // finite sums stay below kInf and acc <= kInf, so acc + time cannot wrap
-                    if (__all_sync(0xffffffffu, lim >= (TM - 1) * 32)) {
+                int32_t* R = stg0 + (s0l + u) * RS + (mm[u] & 3) + col;
+                // finite sums stay below kInf and acc <= kInf, so acc + time cannot wrap
 #pragma unroll
-                        for (int j = 0; j < TM; ++j) po[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
-                    } else {
+                for (int j = 0; j < TM; ++j)
+                    if (j < nj) R[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
+            }
+            if (ms == 0) {
 #pragma unroll
-                        for (int j = 0; j < TM; ++j)
-                            if (j * 32 <= lim) po[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
-                    }
-                    if (is_last) {
-                        int32_t* pl2 = a.C_last + (size_t)i * slice + o;
+                for (int u = 0; u < TS; ++u)
+                    if (lane == u) hdr0[s0l + u] = mm[u];
+                if (sg == 0 && lane == 0) hdr0[SB] = inst;
+            }
+            if (ARG && nj > 0) {
+                const int s0 = pos.sb * SB + s0l;
+                const int base = M - mw - lane;
 #pragma unroll
-                        for (int j = 0; j < TM; ++j)
-                            if (j * 32 <= lim) pl2[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
-                    }
-                    if (ARG) {
-                        uint8_t* pa = a.A + ((size_t)i * a.Lmax + l) * slice + o;
+                for (int u = 0; u < TS; ++u)
+                    if (s0 + u < S) {
+                        const int lim = base - mm[u];
+                        uint8_t* pa = a.A + ((size_t)inst * a.Lmax + l) * slice + (size_t)(s0 + u) * m_pitch + (size_t)(mm[u] + mw + lane);
 #pragma unroll
                         for (int j = 0; j < TM; ++j)
                             if (j * 32 <= lim) pa[j * 32] = (uint8_t)(acc[j][u] >= kInf ? 255 : arg[ARG ? j : 0][ARG ? u : 0]);
                     }
-                }
             }
         }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // staging writes -> visible to the TMA unit
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&out_full);
     }
+}
+
+// C_last[i] = layer L[i]-1 of instance i (from the full table, or from the rolling buffer that
+// layer was written to), 128 bits per thread.
+__global__ void copy_last_kernel(DpArgs a)
+{
+    const int i = blockIdx.y;
+    if (a.status[i] != 0) return;
+    const int Li = a.L[i];
+    const size_t slice = (size_t)a.S * a.m_pitch;
+    const int32_t* src = a.C ? a.C + ((size_t)i * a.Lmax + (Li - 1)) * slice : a.roll + ((size_t)((Li - 1) & 1) * a.B + i) * slice;
+    const int4* s4 = reinterpret_cast<const int4*>(src);
+    int4* d4 = reinterpret_cast<int4*>(a.C_last + (size_t)i * slice);
+    for (size_t k = (size_t)blockIdx.x * blockDim.x + threadIdx.x; k < slice / 4; k += (size_t)gridDim.x * blockDim.x) d4[k] = s4[k];
 }
 
 // Sets the TIMEOUT bit everywhere when a bounded wait ran out.
@@ -539,7 +612,7 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st
 {
     auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG>;
     if (!maps) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
-    kern<<<pl.grid, (NSG * NMS + 2) * 32, pl.smem, st>>>(a, pl, l, maps[0], maps[1]);
+    kern<<<pl.grid, (NSG * NMS + 3) * 32, pl.smem, st>>>(a, pl, l, maps[0], maps[1]);
     return cudaGetLastError();
 }
 
@@ -595,23 +668,29 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     pl->nms = 16 / pl->nsg;
     if (pl->nms < 1) pl->nms = 1;
     pl->tmb = pl->nms * 32 * pl->tm;
-    pl->threads = (pl->nsg * pl->nms + 2) * 32;           // consumer warps + producer + helper
+    pl->threads = (pl->nsg * pl->nms + 3) * 32;           // consumer warps + producer + helper + store warp
     // stages of ks * (tmb + sb) ints: aim at <= 40 KB each, 2..4 of them in the opt-in shared memory
-    const int avail = ctx->smem_optin - 2048 - kMaxStages * (2 * pl->sb + 4) * 4;
+    const int extra = ((kMaxStages * (2 * pl->sb + 4) + 31) & ~31) * 4      // item records
+                      + (pl->sb * (pl->tmb + 4) + pl->sb + 4) * 4;        // staging tile and its header
+    const int avail = ctx->smem_optin - 2048 - extra;
     const int row = (pl->tmb + pl->sb) * 4;
-    int ks = (40 * 1024) / row;
-    if (ks > S) ks = S;
-    if (ks >= 8) ks &= ~7;
-    if (ks < 1) ks = 1;
-    const int stage_bytes = (ks * row + 127) & ~127;
-    int nst = avail / stage_bytes;
+    // chunks of s': as few per item as leave room for two stages (every chunk costs the consumers
+    // a barrier hand-over), of equal size, multiples of 8 rows
+    int nkc = 1, ks = S, stage_bytes = 0, nst = 0;
+    for (;; ++nkc) {
+        ks = (S + nkc - 1) / nkc;
+        if (ks >= 8) ks = (ks + 7) & ~7;
+        stage_bytes = (ks * row + 127) & ~127;
+        nst = avail / stage_bytes;
+        if (nst >= 2 || ks == 1) break;
+    }
     if (nst > kMaxStages) nst = kMaxStages;
     if (nst < 2) return false;
     pl->ks = ks;
     pl->nst = nst;
     pl->nkc = (S + ks - 1) / ks;
     pl->ntiles_m = (sh->M + 1 + pl->tmb - 1) / pl->tmb;
-    pl->smem = nst * stage_bytes + nst * (2 * pl->sb + 4) * 4;
+    pl->smem = nst * stage_bytes + extra;
     pl->tma_t = (S % 4) == 0;                             // trans row pitch a multiple of 16 bytes
     const long long items = (long long)sh->B * pl->ntiles_m * pl->nsb;
     pl->grid = (int)(items < ctx->num_sms ? items : ctx->num_sms);
@@ -706,6 +785,17 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
         if (e != cudaSuccess) return e;
     }
     if (ctx->profiling) { cudaEventRecord(ctx->ev1, st); ctx->ev_valid = 1; }
+    for (int b0 = 0; b0 < B; b0 += 65535) {                   // grid.y limit
+        DpArgs c = a;
+        const int nb = (B - b0 < 65535) ? B - b0 : 65535;
+        c.L += b0; c.status += b0;
+        if (c.C) c.C += (size_t)b0 * Lmax * S * a.m_pitch;
+        c.C_last += (size_t)b0 * S * a.m_pitch;
+        c.roll += (size_t)b0 * S * a.m_pitch;
+        size_t per = ((size_t)S * a.m_pitch / 4 + 255) / 256;
+        if (per > 64) per = 64;
+        copy_last_kernel<<<dim3((unsigned)per, nb), 256, 0, st>>>(c);
+    }
     finalize_kernel<<<(B + 255) / 256, 256, 0, st>>>(B, a.err, a.status);
     return cudaGetLastError();
 }
