@@ -192,6 +192,42 @@ int galv_backtrack(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
                    int32_t* opt_cost, int32_t* plan, int32_t* mem_used,
                    int32_t* status, void* stream);
 
+/*
+ * Outer selection over the instance batch (Section 3: the emitted plan also fixes the number of
+ * pipeline stages and the micro-batch; Section 2: pipelines run with many micro-batches).  Every
+ * instance is one candidate (micro-batch, pipeline degree) whose per-stage optimum opt_cost[i] the
+ * search has found.  An iteration of a pp-stage pipeline fed with n_micro micro-batches lasts
+ * (n_micro + pp - 1) stage times; within each group of candidates (same global batch) the
+ * feasible one (status 0, finite cost) with the shortest iteration wins, the lowest index on ties.
+ * opt_cost, status, n_micro, pp, group: int32 [B]; group values 0..G-1 (others, and n_micro < 1 or
+ * pp < 1, are ignored).  best_time int64 [G] (time units; -1 if the group has no feasible
+ * candidate), best_inst int32 [G] (-1 likewise).  All device pointers.
+ */
+int galv_select_best(galv_ctx* ctx, int32_t B, int32_t G, const int32_t* opt_cost, const int32_t* status,
+                     const int32_t* n_micro, const int32_t* pp, const int32_t* group,
+                     int64_t* best_time, int32_t* best_inst, void* stream);
+
+/*
+ * Dominated-strategy prune (Section 3: a prune of the candidates precedes the dynamic program).
+ * Strategy s is dropped when another strategy d is at least as good in every layer of every
+ * instance of the batch (time and memory) and in every transition (trans(x,d) <= trans(x,s) and
+ * trans(d,x) <= trans(s,x) for all x), and either d < s or d is strictly faster at every layer.
+ * Under this rule the search on the remaining strategies returns the same optimal cost and, after
+ * galv_expand_plan, the same plan as the search on all of them, at every budget.
+ * keep int32 [S]: 1 kept, 0 dropped; map int32 [S]: original indices of the kept strategies in
+ * ascending order, -1 beyond; S_kept int32 [1].  All device pointers; read S_kept back (after
+ * synchronising the stream) to size the compacted tables.  shape.M, m_pitch and flags are not used.
+ */
+int galv_prune_strategies(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                          const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,
+                          int32_t* keep, int32_t* map, int32_t* S_kept, void* stream);
+/* Gather the kept strategies: time_out, mem_out [B][Lmax][S_kept], trans_out [B][S_kept][S_kept]. */
+int galv_compact_tables(galv_ctx* ctx, const galv_shape* shape, int32_t S_kept, const int32_t* map,
+                        const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,
+                        int32_t* time_out, int32_t* mem_out, int32_t* trans_out, void* stream);
+/* Turn a plan over kept strategies back into original indices, in place: plan[e] = map[plan[e]] where >= 0. */
+int galv_expand_plan(galv_ctx* ctx, int32_t B, int32_t Lmax, const int32_t* map, int32_t* plan, void* stream);
+
 /* Bytes of device arena galv_search_host needs (0 on invalid shape). */
 size_t galv_search_host_arena_bytes(const galv_ctx* ctx, const galv_shape* shape, int with_model);
 

@@ -281,3 +281,64 @@ void orc_eval_costs(int L, int S, const orc_layer *layers, const orc_strategy *s
                 trans_q[a * S + c] = orc_quant_time(orc_trans_cost(&layers[0], &strat[a], &strat[c], in),
                                                     in->time_unit_ns);
 }
+
+/* ------------------------------------------------------------------ outer selection
+ *
+ * The plan the selector finally emits also fixes the number of pipeline stages and the
+ * micro-batch (Section 3, "Dynamic Strategy Selector"; Section 2 on pipelines run with many
+ * micro-batches).  Each search instance is one candidate (micro-batch, pipeline degree) whose
+ * per-stage optimum the DP has found; one training iteration of a pp-stage pipeline fed with
+ * n_micro micro-batches lasts (n_micro + pp - 1) stage times (fill and drain).  Within each group
+ * of candidates (same global batch, so the shortest iteration is the highest throughput) pick
+ * the feasible instance with the smallest iteration time, the lowest index on ties.
+ * best_time[g] = -1 and best_inst[g] = -1 when the group has no feasible candidate.
+ * Candidates with n_micro < 1, pp < 1 or a group outside 0..G-1 are ignored.
+ */
+void orc_select_best(int B, int G, const int32_t *opt_cost, const int32_t *status, const int32_t *n_micro,
+                     const int32_t *pp, const int32_t *group, int64_t *best_time, int32_t *best_inst)
+{
+    for (int g = 0; g < G; g++) { best_time[g] = -1; best_inst[g] = -1; }
+    for (int i = 0; i < B; i++) {
+        if (status[i] != 0 || opt_cost[i] >= ORC_INF || opt_cost[i] < 0) continue;
+        if (n_micro[i] < 1 || pp[i] < 1 || group[i] < 0 || group[i] >= G) continue;
+        int64_t t = ((int64_t)n_micro[i] + pp[i] - 1) * (int64_t)opt_cost[i];
+        int g = group[i];
+        if (best_inst[g] < 0 || t < best_time[g]) { best_time[g] = t; best_inst[g] = i; }
+    }
+}
+
+/* ------------------------------------------------------------------ dominated-strategy prune
+ *
+ * The paper prunes the candidate strategies before the dynamic program (Section 3: a decision-tree
+ * prune precedes the search).  The rule here is the one that provably leaves the search result
+ * untouched, plan included: strategy s goes when some other strategy d is at least as good in every
+ * respect, in every instance of the batch -
+ *    time(l,d) <= time(l,s) and mem(l,d) <= mem(l,s) for every layer l < L,
+ *    trans(x,d) <= trans(x,s) and trans(d,x) <= trans(s,x) for every strategy x -
+ * and either d < s (then swapping s for d in a plan never costs more and makes the plan smaller in
+ * the (p_{L-1},..,p_0) order, so the reported plan never holds s), or d is strictly faster at every
+ * layer (then a plan holding s is never optimal).  keep[s] = 1 for the survivors.
+ */
+void orc_prune(int B, int Lmax, int S, const int32_t *L, const int32_t *time, const int32_t *mem,
+               const int32_t *trans, int32_t *keep)
+{
+    for (int s = 0; s < S; s++) {
+        keep[s] = 1;
+        for (int d = 0; d < S && keep[s]; d++) {
+            if (d == s) continue;
+            int dominated = 1, strict = 1;
+            for (int i = 0; i < B && dominated; i++) {
+                if (L[i] < 1 || L[i] > Lmax) continue;
+                const int32_t *t = time + (int64_t)i * Lmax * S, *m = mem + (int64_t)i * Lmax * S;
+                const int32_t *x = trans + (int64_t)i * S * S;
+                for (int l = 0; l < L[i]; l++) {
+                    if (t[l * S + d] > t[l * S + s] || m[l * S + d] > m[l * S + s]) { dominated = 0; break; }
+                    if (t[l * S + d] >= t[l * S + s]) strict = 0;
+                }
+                for (int k = 0; k < S && dominated; k++)
+                    if (x[k * S + d] > x[k * S + s] || x[d * S + k] > x[s * S + k]) dominated = 0;
+            }
+            if (dominated && (d < s || strict)) keep[s] = 0;
+        }
+    }
+}

@@ -128,3 +128,20 @@ def search(time, mem, trans, M: int, budget=None, use_A: bool = False):
     Ct, At = dp(time, mem, trans, M, want_A=True)
     opt, plan, used, st2 = backtrack(time, mem, trans, Ct, At if use_A else None, M if budget is None else budget)
     return dict(status=st | st2, opt_cost=opt, plan=plan, mem_used=used, C=Ct, A=At)
+
+
+def select_best(opt_cost, status, n_micro, pp, group, G: int):
+    """(best_time int64 [G], best_inst int32 [G]): per group the feasible candidate with the shortest iteration."""
+    oc, p0 = _i32(opt_cost); st, p1 = _i32(status); nm, p2 = _i32(n_micro); ppa, p3 = _i32(pp); gr, p4 = _i32(group)
+    bt = np.empty(G, np.int64); bi = np.empty(G, np.int32)
+    lib().orc_select_best(len(oc), G, p0, p1, p2, p3, p4, bt.ctypes.data_as(C.c_void_p), bi.ctypes.data_as(C.c_void_p))
+    return bt, bi
+
+
+def prune(L, time, mem, trans):
+    """keep[S] (0/1): strategies that survive the dominated-strategy prune over the whole batch."""
+    time, pt = _i32(time); mem, pm = _i32(mem); trans, px = _i32(trans); L, pl = _i32(L)
+    B, Lmax, S = time.shape
+    keep = np.empty(S, np.int32)
+    lib().orc_prune(B, Lmax, S, pl, pt, pm, px, keep.ctypes.data_as(C.c_void_p))
+    return keep

@@ -23,7 +23,8 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgalv.so"
 
 EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "galv_eval_costs",
            "galv_dp_workspace_bytes", "galv_dp_search", "galv_backtrack", "galv_search_host_arena_bytes",
-           "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_dp_search_static")
+           "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_dp_search_static", "galv_select_best", "galv_prune_strategies",
+           "galv_compact_tables", "galv_expand_plan")
 
 
 class galv_shape(C.Structure):
@@ -62,6 +63,10 @@ def load_library() -> C.CDLL:
     lib.galv_dp_search.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.galv_backtrack.argtypes = [vp, shp] + [vp] * 13
     lib.galv_dp_search_static.argtypes = [vp, shp] + [vp] * 9
+    lib.galv_select_best.argtypes = [vp, C.c_int32, C.c_int32] + [vp] * 8
+    lib.galv_prune_strategies.argtypes = [vp, shp] + [vp] * 8
+    lib.galv_compact_tables.argtypes = [vp, shp, C.c_int32] + [vp] * 8
+    lib.galv_expand_plan.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, vp]
     lib.galv_search_host_arena_bytes.argtypes = [vp, shp, C.c_int]
     lib.galv_search_host_arena_bytes.restype = sz
     lib.galv_search_host.argtypes = [vp, shp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -134,6 +139,21 @@ class Galv:
         self._check(self.lib.galv_dp_search_static(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q),
                                                    _ptr(trans_q), _ptr(Ct), _ptr(At), _ptr(C_last), _ptr(status),
                                                    _stream()))
+
+    def galv_select_best(self, B, G, opt_cost, status, n_micro, pp, group, best_time, best_inst):
+        self._check(self.lib.galv_select_best(self.h, B, G, _ptr(opt_cost), _ptr(status), _ptr(n_micro), _ptr(pp),
+                                              _ptr(group), _ptr(best_time), _ptr(best_inst), _stream()))
+
+    def galv_prune_strategies(self, shape, L, time_q, mem_q, trans_q, keep, map_, S_kept):
+        self._check(self.lib.galv_prune_strategies(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),
+                                                   _ptr(keep), _ptr(map_), _ptr(S_kept), _stream()))
+
+    def galv_compact_tables(self, shape, S_kept, map_, time_q, mem_q, trans_q, time_out, mem_out, trans_out):
+        self._check(self.lib.galv_compact_tables(self.h, C.byref(shape), S_kept, _ptr(map_), _ptr(time_q), _ptr(mem_q),
+                                                 _ptr(trans_q), _ptr(time_out), _ptr(mem_out), _ptr(trans_out), _stream()))
+
+    def galv_expand_plan(self, B, Lmax, map_, plan):
+        self._check(self.lib.galv_expand_plan(self.h, B, Lmax, _ptr(map_), _ptr(plan), _stream()))
 
     def galv_backtrack(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, budget, opt_cost, plan, mem_used, status):
         self._check(self.lib.galv_backtrack(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),
