@@ -60,6 +60,7 @@ extern "C" {
 #define GALV_STORE_C_FULL 1 /* keep every layer of C (needed to backtrack without A) */
 #define GALV_STORE_ARGMIN 2 /* write the argmin table A */
 #define GALV_KERNEL_REFERENCE 256 /* run the recurrence with the simple one-thread-per-cell kernel (slow; cross-checks) */
+#define GALV_KERNEL_PER_LAYER 512 /* one launch per layer instead of one cooperative launch over all layers */
 
 typedef struct galv_ctx galv_ctx;
 
@@ -135,8 +136,10 @@ size_t galv_dp_workspace_bytes(const galv_ctx* ctx, const galv_shape* shape);
  * Pad columns M < m < m_pitch are written as GALV_INF / 255.
  * workspace: 256-byte aligned, at least galv_dp_workspace_bytes(shape) bytes,
  * overwritten by every call (calls sharing a workspace must not overlap).
- * Enqueues one small launch per layer; nothing synchronises the host, so the
- * call may be captured in a CUDA graph.
+ * With the full table and no argmin table all layers run in ONE cooperative launch (its CTAs hand
+ * finished tiles to one another through counters in the workspace, with bounded
+ * waits); otherwise, or with GALV_KERNEL_PER_LAYER, one launch per layer.
+ * Nothing synchronises the host, so the call may be captured in a CUDA graph.
  */
 int galv_dp_search(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
                    const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,

@@ -54,6 +54,15 @@ __device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t by
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all_but_last() { asm volatile("cp.async.bulk.wait_group 1;" ::: "memory"); }
+__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_gpu_add(int32_t* p, int v) {
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -82,14 +91,15 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 // ---------------------------------------------------------------- validation / schedule
 
 // One CTA per instance: entries >= 0, L in range, worst-case path sum below kInf.
-__global__ void validate_kernel(int B, int Lmax, int S, const int32_t* __restrict__ L,
+__global__ void validate_kernel(int B, int Lmax, int S, int M, const int32_t* __restrict__ L,
                                 const int32_t* __restrict__ time_q, const int32_t* __restrict__ mem_q,
-                                const int32_t* __restrict__ trans_q, int32_t* __restrict__ status)
+                                const int32_t* __restrict__ trans_q, int32_t* __restrict__ status,
+                                int32_t* __restrict__ maxmem)
 {
     const int i = blockIdx.x;
     __shared__ long long s_sum;
-    __shared__ int s_tmax, s_bad;
-    if (threadIdx.x == 0) { s_sum = 0; s_tmax = 0; s_bad = 0; }
+    __shared__ int s_tmax, s_bad, s_mmax;
+    if (threadIdx.x == 0) { s_sum = 0; s_tmax = 0; s_bad = 0; s_mmax = 0; }
     __syncthreads();
     const int Li = L[i];
     if (Li < 1 || Li > Lmax) {
@@ -97,7 +107,7 @@ __global__ void validate_kernel(int B, int Lmax, int S, const int32_t* __restric
         return;
     }
     long long sum = 0;
-    int bad = 0, tmax = 0;
+    int bad = 0, tmax = 0, mmax = 0;
     const int32_t* t = time_q + (size_t)i * Lmax * S;
     const int32_t* mq = mem_q + (size_t)i * Lmax * S;
     for (int l = threadIdx.x; l < Li; l += blockDim.x) {
@@ -106,6 +116,7 @@ __global__ void validate_kernel(int B, int Lmax, int S, const int32_t* __restric
             const int tv = t[l * S + s], mv = mq[l * S + s];
             bad |= (tv < 0) | (mv < 0);
             mx = max(mx, tv);
+            mmax = max(mmax, mv);
         }
         sum += mx;
     }
@@ -117,6 +128,7 @@ __global__ void validate_kernel(int B, int Lmax, int S, const int32_t* __restric
     }
     atomicAdd(reinterpret_cast<unsigned long long*>(&s_sum), static_cast<unsigned long long>(sum));
     atomicMax(&s_tmax, tmax);
+    atomicMax(&s_mmax, mmax);
     if (bad) atomicOr(&s_bad, 1);
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -124,6 +136,8 @@ __global__ void validate_kernel(int B, int Lmax, int S, const int32_t* __restric
         if (s_bad) st = GALV_STATUS_BAD_INPUT;
         else if (s_sum + (long long)(Li - 1) * s_tmax >= (long long)kInf) st = GALV_STATUS_OVERFLOW_RISK;
         status[i] = st;
+        // largest shift of a stored row over the valid instances (M+1 stands for "fills the whole row")
+        if (st == 0) atomicMax(maxmem, min(s_mmax, M + 1));
     }
 }
 
@@ -255,8 +269,8 @@ __device__ __forceinline__ long long item_at_weight(long long target, const DpPl
     return oi * pl.ntiles_m * pl.nsb + idx;
 }
 
-template <int TM, int NSG, int NMS, bool ARG>
-__global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l,
+template <int TM, int NSG, int NMS, bool ARG, bool MULTI>
+__global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
                                                                               const __grid_constant__ CUtensorMap map_t)
 {
@@ -273,19 +287,28 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
     __shared__ __align__(8) uint64_t out_full, out_empty;  // staging tile written / drained
+    __shared__ int fill_count;                             // helper -> store warp: first tiles whose unreachable cells are written
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
     const int KS = pl.ks, NKC = pl.nkc, NST = pl.nst;
+    const int l_last = MULTI ? l_last_arg : l_first + 1;  // single-layer instantiation: loops over l run once
+    int32_t* const tile_done = MULTI ? a.tile_done : nullptr;
 
-    const int nact = a.nactive[l];
-    // weight of the last tile of an instance: its 32-column groups out of TMB/32, in 64ths
+    // Layers l_first .. l_last-1.  One layer per launch, or all of them in one cooperative launch
+    // (a.tile_done set): then an item of layer l starts once the tiles of layer l-1 it reads are
+    // complete, which their store warps publish in a.tile_done (see the producer and the store warp).
+    // Every role walks the same sequence of (layer, item); this CTA's items of layer l:
     const int last_cols = M + 1 - (pl.ntiles_m - 1) * TMB;
+    // weight of the last tile of an instance: its 32-column groups out of TMB/32, in 64ths
     const int wr = max(1, ((last_cols + 31) / 32) * 64 / (TMB / 32));
-    const long long wtot = (long long)nact * pl.nsb * ((long long)(pl.ntiles_m - 1) * 64 + wr);
-    const long long it0 = item_at_weight(wtot * blockIdx.x / gridDim.x, pl, wr);
-    const long long it1 = item_at_weight(wtot * (blockIdx.x + 1) / gridDim.x, pl, wr);
-    if (it0 >= it1) return;
+    auto layer_range = [&](int l, ItemPos& first) -> int {          // first item and how many
+        const long long wtot = (long long)a.nactive[l] * pl.nsb * ((long long)(pl.ntiles_m - 1) * 64 + wr);
+        const long long it0 = item_at_weight(wtot * blockIdx.x / gridDim.x, pl, wr);
+        const long long it1 = item_at_weight(wtot * (blockIdx.x + 1) / gridDim.x, pl, wr);
+        first = item_at(it0, pl);
+        return (int)(it1 - it0);
+    };
 
     // stage: NBOX boxes of [KS][BOXC] previous-layer values, then [KS][SB] trans values; 128-byte multiples
     int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
@@ -299,22 +322,49 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         for (int k = 0; k < NST; ++k) { mbar_init(&full_bar[k], 2); mbar_init(&empty_bar[k], NC); }
         mbar_init(&out_full, NC);
         mbar_init(&out_empty, 1);
+        fill_count = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
     const size_t slice = (size_t)S * m_pitch;
-    ItemPos pos = item_at(it0, pl);
 
     if (warp == NC) {
         // ------------------------------------------------------------ producer
         const bool tma_t = pl.tma_t != 0;                 // trans rows 16-byte aligned: one box per chunk
-        const int row0 = a.C ? (l - 1) * S : ((l - 1) & 1) * a.B * S;      // row of (instance 0, layer l-1, s'=0)
         const int inst_rows = a.C ? a.Lmax * S : S;
+        // tiles of the previous layer an item reads: its own and, because rows are stored shifted by
+        // up to the largest mem, the kdep before it
+        const int kdep = tile_done ? (min(*a.maxmem, M) + TMB - 1) / TMB : 0;
         int n = 0;                                        // chunk counter
-        for (long long item = it0; item < it1; ++item, item_next(pos, pl)) {
+        for (int l = l_first; l < l_last; ++l) {
+        ItemPos pos;
+        const int nit = layer_range(l, pos);
+        const int row0 = a.C ? (l - 1) * S : ((l - 1) & 1) * a.B * S;      // row of (instance 0, layer l-1, s'=0)
+        for (int q = 0; q < nit; ++q, item_next(pos, pl)) {
             const int i = a.order[pos.oi];
             const int m0 = pos.mt * TMB;
+            if (MULTI && tile_done && l > 1) {
+                // bounded wait for the tiles of layer l-1 (all their s-blocks) this item reads
+                const int need = (l - 1) * pl.nsb;
+                bool ok = true;
+                if (lane == 0) {
+                    for (int t = max(0, pos.mt - kdep); t <= pos.mt && ok; ++t) {
+                        const int32_t* c = tile_done + (size_t)i * pl.ntiles_m + t;
+                        int spins = 0;
+                        while (ld_acquire_gpu(c) < need) {
+                            if (++spins > kSpinLimit) { ok = false; break; }
+                            __nanosleep(64);
+                        }
+                    }
+                    asm volatile("fence.proxy.async;" ::: "memory");     // what was acquired -> visible to the TMA loads below
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+            }
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
             const int yc = row0 + i * inst_rows;
@@ -348,12 +398,16 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 __syncwarp();
             }
         }
+        }
         return;
     }
     if (warp == NC + 1) {
         // ------------------------------------------------------------ helper
         int n = 0;
-        for (long long item = it0; item < it1; ++item, item_next(pos, pl)) {
+        for (int l = l_first; l < l_last; ++l) {
+        ItemPos pos;
+        const int nit = layer_range(l, pos);
+        for (int q = 0; q < nit; ++q, item_next(pos, pl)) {
             const int i = a.order[pos.oi];
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);
@@ -392,7 +446,14 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                         if (ARG) aout[o + mm] = 255;
                     }
                 }
+                if (MULTI && tile_done) {
+                    // the store warp publishes the tile; it must know these cells are out
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) atomicAdd(&fill_count, 1);      // a counter, not a barrier phase: the helper may be several first tiles ahead
+                }
             }
+        }
         }
         return;
     }
@@ -404,7 +465,21 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         // table columns above M do not exist.  Each lane takes rows lane, lane+32: the 16-byte aligned
         // middle leaves as one bulk store, the few cells before and after it as plain stores.
         int it = 0;
-        for (long long item = it0; item < it1; ++item, item_next(pos, pl), ++it) {
+        int32_t* unpublished = nullptr;                   // tile counter of the previous item, not yet bumped
+        int nfill = 0;                                    // first tiles seen so far
+        // Publishing a tile: its bulk stores complete, every lane's plain stores fenced, one release add.
+        auto publish = [&](int32_t* counter) {
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) {
+                asm volatile("fence.proxy.async;" ::: "memory");
+                red_release_gpu_add(counter, 1);
+            }
+        };
+        for (int l = l_first; l < l_last; ++l) {
+        ItemPos pos;
+        const int nit = layer_range(l, pos);
+        for (int q = 0; q < nit; ++q, item_next(pos, pl), ++it) {
             if (!mbar_wait(&out_full, it & 1)) {
                 if (lane == 0) atomicExch(a.err, 1);
                 return;
@@ -432,6 +507,28 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
             bulk_wait_read();                                     // the staging tile may be overwritten
             __syncwarp();
             if (lane == 0) mbar_arrive(&out_empty);
+            if (MULTI && tile_done) {
+                // The previous item's bulk stores were issued a whole item ago: waiting for all groups
+                // but the newest costs nothing, and then that item is published.  The last item of a
+                // layer is published at once: other CTAs' first items of the next layer may need it,
+                // and this CTA's own next item may in turn wait for theirs.
+                int32_t* mine = tile_done + (size_t)i * pl.ntiles_m + pos.mt;
+                if (pos.mt == 0) {                                // the helper's fill of this tile (it runs ahead)
+                    ++nfill;
+                    int spins = 0;
+                    while (*reinterpret_cast<volatile int*>(&fill_count) < nfill) {
+                        if (++spins > kSpinLimit) {
+                            if (lane == 0) atomicExch(a.err, 1);
+                            return;
+                        }
+                        __nanosleep(64);
+                    }
+                }
+                if (unpublished) { bulk_wait_all_but_last(); publish(unpublished); }
+                if (q + 1 == nit) { bulk_wait_all(); publish(mine); unpublished = nullptr; }
+                else unpublished = mine;
+            }
+        }
         }
         bulk_wait_all();
         return;
@@ -442,8 +539,11 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
     int acc[TM][TS];
     int arg[ARG ? TM : 1][ARG ? TS : 1];
     (void)arg;
-    int n = 0;
-    for (long long item = it0; item < it1; ++item, item_next(pos, pl)) {
+    int n = 0, it = 0;
+    for (int l = l_first; l < l_last; ++l) {
+    ItemPos pos;
+    const int nit = layer_range(l, pos);
+    for (int q = 0; q < nit; ++q, item_next(pos, pl), ++it) {
         const int mw = pos.mt * TMB + ms * (32 * TM);       // first column of this warp
         // 32-column groups of this warp that hold at least one column <= M
         const int nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
@@ -543,7 +643,6 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
 
         // Epilogue: add time(l,s) and hand the tile to the store warps through the staging tile;
         // row s is written shifted by mem(l,s) mod 4 (see the store warps).
-        const int it = (int)(item - it0);
         if (it > 0 && !mbar_wait(&out_empty, (it - 1) & 1)) {    // the previous item has been drained
             if (lane == 0) atomicExch(a.err, 1);
             return;
@@ -583,6 +682,7 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         __syncwarp();
         if (lane == 0) mbar_arrive(&out_full);
     }
+    }
 }
 
 // C_last[i] = layer L[i]-1 of instance i (from the full table, or from the rolling buffer that
@@ -607,28 +707,40 @@ __global__ void finalize_kernel(int B, const int32_t* err, int32_t* status)
         status[i] |= GALV_STATUS_TIMEOUT;
 }
 
+// maps == nullptr: only opt the instantiation into its dynamic shared memory.  Layers l_first..l_last-1;
+// more than one layer means the CTAs wait on one another's tiles, so the launch is cooperative
+// (all CTAs guaranteed co-resident).
 template <int TM, int NSG, int NMS, bool ARG>
-cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st, const CUtensorMap* maps)
+cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_last, cudaStream_t st, const CUtensorMap* maps)
 {
-    auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG>;
-    if (!maps) return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
-    kern<<<pl.grid, (NSG * NMS + 3) * 32, pl.smem, st>>>(a, pl, l, maps[0], maps[1]);
+    auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG, false>;
+    auto kern_multi = layer_tiled_kernel<TM, NSG, NMS, false, true>;
+    if (!maps) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+        if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_multi, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+        return e;
+    }
+    if (l_last - l_first > 1) {
+        void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[0], (void*)&maps[1]};
+        return cudaLaunchCooperativeKernel((const void*)kern_multi, dim3(pl.grid), dim3((NSG * NMS + 3) * 32), args, (size_t)pl.smem, st);
+    }
+    kern<<<pl.grid, (NSG * NMS + 3) * 32, pl.smem, st>>>(a, pl, l_first, l_last, maps[0], maps[1]);
     return cudaGetLastError();
 }
 
 // nsg warps along s, 16/nsg (rounded down) along m: one instantiation per s-block width.
 template <bool ARG>
-cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l, cudaStream_t st, const CUtensorMap* maps)
+cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l_first, int l_last, cudaStream_t st, const CUtensorMap* maps)
 {
     switch (pl.nsg) {
-    case 1: return launch_one<4, 1, 16, ARG>(a, pl, l, st, maps);
-    case 2: return launch_one<4, 2, 8, ARG>(a, pl, l, st, maps);
-    case 3: return launch_one<4, 3, 5, ARG>(a, pl, l, st, maps);
-    case 4: return launch_one<4, 4, 4, ARG>(a, pl, l, st, maps);
-    case 5: return launch_one<4, 5, 3, ARG>(a, pl, l, st, maps);
-    case 6: return launch_one<4, 6, 2, ARG>(a, pl, l, st, maps);
-    case 7: return launch_one<4, 7, 2, ARG>(a, pl, l, st, maps);
-    case 8: return launch_one<4, 8, 2, ARG>(a, pl, l, st, maps);
+    case 1: return launch_one<4, 1, 16, ARG>(a, pl, l_first, l_last, st, maps);
+    case 2: return launch_one<4, 2, 8, ARG>(a, pl, l_first, l_last, st, maps);
+    case 3: return launch_one<4, 3, 5, ARG>(a, pl, l_first, l_last, st, maps);
+    case 4: return launch_one<4, 4, 4, ARG>(a, pl, l_first, l_last, st, maps);
+    case 5: return launch_one<4, 5, 3, ARG>(a, pl, l_first, l_last, st, maps);
+    case 6: return launch_one<4, 6, 2, ARG>(a, pl, l_first, l_last, st, maps);
+    case 7: return launch_one<4, 7, 2, ARG>(a, pl, l_first, l_last, st, maps);
+    case 8: return launch_one<4, 8, 2, ARG>(a, pl, l_first, l_last, st, maps);
     default: return cudaErrorInvalidConfiguration;
     }
 }
@@ -650,7 +762,8 @@ WsLayout galv_ws_layout(const galv_shape* sh)
     w.order = off;   off = align256(off + (size_t)sh->B * 4);
     w.nactive = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.scratch = off; off = align256(off + (size_t)2 * (sh->Lmax + 2) * 4);
-    w.err = off;     off = align256(off + 4);
+    w.err = off;     off = align256(off + 8);                  // error flag, largest mem
+    w.tile_done = off; off = align256(off + (size_t)sh->B * ((sh->M + 128) / 128) * 4);   // per (instance, tile of >= 128 columns)
     w.roll = off;
     if (!(sh->flags & GALV_STORE_C_FULL)) off = align256(off + (size_t)2 * sh->B * sh->S * sh->m_pitch * 4);
     w.total = off;
@@ -726,8 +839,8 @@ cudaError_t galv_dp_configure(const galv_ctx* ctx)
     pl.smem = ctx->smem_optin - 2048;
     for (int nsg = 1; nsg <= 8; ++nsg) {
         pl.nsg = nsg;
-        cudaError_t e = launch_tiled<false>(a, pl, 0, nullptr, nullptr);
-        if (e == cudaSuccess) e = launch_tiled<true>(a, pl, 0, nullptr, nullptr);
+        cudaError_t e = launch_tiled<false>(a, pl, 0, 0, nullptr, nullptr);
+        if (e == cudaSuccess) e = launch_tiled<true>(a, pl, 0, 0, nullptr, nullptr);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -739,9 +852,9 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     const int B = a.B, Lmax = a.Lmax, S = a.S;
     e = cudaMemsetAsync(a.scratch, 0, (size_t)2 * (Lmax + 2) * 4, st);
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(a.err, 0, 4, st);
+    e = cudaMemsetAsync(a.err, 0, 8, st);
     if (e != cudaSuccess) return e;
-    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.L, a.time_q, a.mem_q, a.trans_q, a.status);
+    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1);
     schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.L, a.status, a.order, a.nactive, a.scratch);
     {
         int gx = (a.m_pitch + 255) / 256;
@@ -773,14 +886,28 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
         if (pl.tma_t &&
             (e = encode_2d(&maps[1], (void*)a.trans_q, (size_t)S, (size_t)B * S, pl.sb, pl.ks)) != cudaSuccess) return e;
     }
+    // All layers in one cooperative launch when the grid's CTAs can be co-resident (they wait on one
+    // another's tiles); with an argmin table, on request, or for the reference kernel: one launch per layer.
+    // (with the two-layer rolling buffer a layer would overwrite cells a slower CTA still reads)
+    const bool persistent = !reference && a.C && !a.A && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
+    DpArgs ap = a;
+    ap.tile_done = nullptr;
+    ap.maxmem = a.err + 1;
+    if (persistent) {
+        ap.tile_done = a.tile_done;
+        if ((e = cudaMemsetAsync(a.tile_done, 0, (size_t)B * pl.ntiles_m * 4, st)) != cudaSuccess) return e;
+    }
     if (ctx->profiling) cudaEventRecord(ctx->ev0, st);
-    for (int l = 1; l < Lmax; ++l) {
+    if (persistent) {
+        if ((e = launch_tiled<false>(ap, pl, 1, Lmax, st, maps)) != cudaSuccess) return e;
+    }
+    for (int l = 1; l < Lmax && !persistent; ++l) {
         if (reference) {
             const int mchunks = (a.m_pitch + 255) / 256;
             layer_reference_kernel<<<dim3((unsigned)((size_t)B * mchunks), S, 1), 256, 0, st>>>(a, l);
             e = cudaGetLastError();
         } else {
-            e = a.A ? launch_tiled<true>(a, pl, l, st, maps) : launch_tiled<false>(a, pl, l, st, maps);
+            e = a.A ? launch_tiled<true>(ap, pl, l, l + 1, st, maps) : launch_tiled<false>(ap, pl, l, l + 1, st, maps);
         }
         if (e != cudaSuccess) return e;
     }

@@ -49,6 +49,8 @@ struct DpArgs {
     int32_t* nactive;    // [Lmax+1] instances with L > l
     int32_t* scratch;    // [2*(Lmax+2)] histogram / fill counters
     int32_t* err;        // device error flag
+    int32_t* tile_done;  // [B][ntiles_m] finished items per (instance, tile); NULL when layers are separate launches
+    int32_t* maxmem;     // largest mem over the valid instances (min(.., M+1))
     int32_t* status;
 };
 
@@ -56,7 +58,7 @@ struct DpArgs {
 int galv_set_error(galv_ctx* ctx, int code, const char* text);
 
 // workspace carve-up (offsets in bytes, all 256-aligned)
-struct WsLayout { size_t order, nactive, scratch, err, roll, total; };
+struct WsLayout { size_t order, nactive, scratch, err, tile_done, roll, total; };
 WsLayout galv_ws_layout(const galv_shape* sh);
 
 bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* plan);

@@ -88,7 +88,8 @@ def check_batch(orc, galv, w, flags, idx=None, tables=True, budget=None):
     return sb, res
 
 
-MODES = [1, 3, 2, 1 | 256, 3 | 256]      # full C; full C + A; rolling + A; the same with the reference kernel
+MODES = [1, 3, 2, 1 | 512, 1 | 256, 3 | 256]   # full C (all layers in one launch); full C + A; rolling + A;
+                                             # full C with one launch per layer; the reference kernel
 
 
 @pytest.mark.parametrize("flags", MODES)
@@ -121,7 +122,7 @@ SHAPES = [  # B, Lmax, S, M, kwargs
 ]
 
 
-@pytest.mark.parametrize("flags", [1, 3, 2])
+@pytest.mark.parametrize("flags", [1, 3, 2, 1 | 512])
 @pytest.mark.parametrize("k", range(len(SHAPES)))
 def test_random_shapes(orc, galv, flags, k):
     B, Lmax, S, M, kw = SHAPES[k]
