@@ -55,9 +55,9 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all_but_last() { asm volatile("cp.async.bulk.wait_group 1;" ::: "memory"); }
-__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
+__device__ __forceinline__ int ld_relaxed_gpu(const int32_t* p) {
     int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ void red_release_gpu_add(int32_t* p, int v) {
@@ -347,19 +347,23 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
             if (MULTI && tile_done && l > 1) {
                 // bounded wait for the tiles of layer l-1 (all their s-blocks) this item reads
                 const int need = (l - 1) * pl.nsb;
+                // one lane per tile polls (relaxed), then one acquire fence for the warp
                 bool ok = true;
-                if (lane == 0) {
-                    for (int t = max(0, pos.mt - kdep); t <= pos.mt && ok; ++t) {
+                for (int t0 = max(0, pos.mt - kdep); t0 <= pos.mt && ok; t0 += 32) {
+                    const int t = t0 + lane;
+                    if (t <= pos.mt) {
                         const int32_t* c = tile_done + (size_t)i * pl.ntiles_m + t;
                         int spins = 0;
-                        while (ld_acquire_gpu(c) < need) {
+                        while (ld_relaxed_gpu(c) < need) {
                             if (++spins > kSpinLimit) { ok = false; break; }
                             __nanosleep(64);
                         }
                     }
-                    asm volatile("fence.proxy.async;" ::: "memory");     // what was acquired -> visible to the TMA loads below
+                    ok = __all_sync(0xffffffffu, ok);
                 }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
+                __threadfence();                                         // acquire: the tiles' data is ordered after the counters
+                asm volatile("fence.proxy.async;" ::: "memory");         // ... and visible to the TMA loads below
+                __syncwarp();
                 if (!ok) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
