@@ -94,7 +94,7 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 __global__ void validate_kernel(int B, int Lmax, int S, int M, const int32_t* __restrict__ L,
                                 const int32_t* __restrict__ time_q, const int32_t* __restrict__ mem_q,
                                 const int32_t* __restrict__ trans_q, int32_t* __restrict__ status,
-                                int32_t* __restrict__ maxmem)
+                                int32_t* __restrict__ maxmem, int32_t* __restrict__ minmem_l)
 {
     const int i = blockIdx.x;
     __shared__ long long s_sum;
@@ -138,13 +138,25 @@ __global__ void validate_kernel(int B, int Lmax, int S, int M, const int32_t* __
         status[i] = st;
         // largest shift of a stored row over the valid instances (M+1 stands for "fills the whole row")
         if (st == 0) atomicMax(maxmem, min(s_mmax, M + 1));
+        s_bad = st;
     }
+    __syncthreads();
+    if (s_bad == 0)
+        for (int l = threadIdx.x; l < Li; l += blockDim.x) {      // smallest mem of each layer over the valid instances
+            int mn = 0x7fffffff;
+            for (int s = 0; s < S; ++s) mn = min(mn, mq[l * S + s]);
+            atomicMin(&minmem_l[l], mn);
+        }
 }
 
 // Single CTA: nactive[l] = valid instances with L > l; order = valid instances, longest first.
 // scratch = hist[Lmax+2] | fill[Lmax+2], zeroed by the host before the launch.
-__global__ void schedule_kernel(int B, int Lmax, const int32_t* __restrict__ L, const int32_t* __restrict__ status,
-                                int32_t* __restrict__ order, int32_t* __restrict__ nactive, int32_t* __restrict__ scratch)
+// ntiles[l] = tiles of tmb columns per instance that can store anything in layer l: column m' lands at
+// m' + mem(l,s) <= M, so tiles starting above M - (smallest mem of the layer) are left out (at least one
+// tile stays: it also writes the cells no column maps to).
+__global__ void schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, const int32_t* __restrict__ L,
+                                const int32_t* __restrict__ status, int32_t* __restrict__ order, int32_t* __restrict__ nactive,
+                                int32_t* __restrict__ scratch, const int32_t* __restrict__ minmem_l, int32_t* __restrict__ ntiles)
 {
     int32_t* hist = scratch;
     int32_t* fill = scratch + Lmax + 2;
@@ -161,6 +173,11 @@ __global__ void schedule_kernel(int B, int Lmax, const int32_t* __restrict__ L, 
             const int Li = L[i];
             order[nactive[Li] + atomicAdd(&fill[Li], 1)] = i;   // instances longer than Li come first
         }
+    for (int l = threadIdx.x; l <= Lmax; l += blockDim.x) {
+        int nt = 1;
+        if (l < Lmax && minmem_l[l] <= M) nt = min(ntiles_m, (M - minmem_l[l]) / tmb + 1);
+        ntiles[l] = max(1, nt);
+    }
 }
 
 // ---------------------------------------------------------------- base layer
@@ -240,17 +257,18 @@ constexpr int kMaxStages = 4;
 
 struct ItemPos { int oi, mt, sb; };
 
-__device__ __forceinline__ ItemPos item_at(long long item, const DpPlan& pl) {
-    const int per = pl.ntiles_m * pl.nsb;
+// nt = tiles per instance in the layer at hand (the trailing tiles that cannot store anything are left out)
+__device__ __forceinline__ ItemPos item_at(long long item, int nt, int nsb) {
+    const int per = nt * nsb;
     ItemPos p;
     p.oi = (int)(item / per);
     const int r = (int)(item - (long long)p.oi * per);
-    p.mt = r / pl.nsb;
-    p.sb = r - p.mt * pl.nsb;
+    p.mt = r / nsb;
+    p.sb = r - p.mt * nsb;
     return p;
 }
-__device__ __forceinline__ void item_next(ItemPos& p, const DpPlan& pl) {
-    if (++p.sb == pl.nsb) { p.sb = 0; if (++p.mt == pl.ntiles_m) { p.mt = 0; ++p.oi; } }
+__device__ __forceinline__ void item_next(ItemPos& p, int nt, int nsb) {
+    if (++p.sb == nsb) { p.sb = 0; if (++p.mt == nt) { p.mt = 0; ++p.oi; } }
 }
 
 // Shared memory: NST stages of [KS][TMB] previous-layer values + [KS][SB] trans values, then per
@@ -260,13 +278,13 @@ __device__ __forceinline__ void item_next(ItemPos& p, const DpPlan& pl) {
 // Items are dealt to CTAs by weight, not by count: a full tile weighs 64, the ragged last tile of
 // an instance (fewer than TMB columns) in proportion to its 32-column groups.  Returns the first
 // item whose cumulative weight reaches `target`.
-__device__ __forceinline__ long long item_at_weight(long long target, const DpPlan& pl, int wr) {
-    const long long full = (long long)(pl.ntiles_m - 1) * pl.nsb * 64;     // weight of an instance's full tiles
-    const long long per = full + (long long)pl.nsb * wr;
+__device__ __forceinline__ long long item_at_weight(long long target, int nt, int nsb, int wr) {
+    const long long full = (long long)(nt - 1) * nsb * 64;                 // weight of an instance's full tiles
+    const long long per = full + (long long)nsb * wr;
     const long long oi = target / per;
     const long long rem = target - oi * per;
-    const long long idx = rem < full ? (rem + 63) / 64 : (pl.ntiles_m - 1) * pl.nsb + (rem - full + wr - 1) / wr;
-    return oi * pl.ntiles_m * pl.nsb + idx;
+    const long long idx = rem < full ? (rem + 63) / 64 : (nt - 1) * nsb + (rem - full + wr - 1) / wr;
+    return oi * nt * nsb + idx;
 }
 
 template <int TM, int NSG, int NMS, bool ARG, bool MULTI>
@@ -299,14 +317,15 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
     // (a.tile_done set): then an item of layer l starts once the tiles of layer l-1 it reads are
     // complete, which their store warps publish in a.tile_done (see the producer and the store warp).
     // Every role walks the same sequence of (layer, item); this CTA's items of layer l:
-    const int last_cols = M + 1 - (pl.ntiles_m - 1) * TMB;
-    // weight of the last tile of an instance: its 32-column groups out of TMB/32, in 64ths
-    const int wr = max(1, ((last_cols + 31) / 32) * 64 / (TMB / 32));
-    auto layer_range = [&](int l, ItemPos& first) -> int {          // first item and how many
-        const long long wtot = (long long)a.nactive[l] * pl.nsb * ((long long)(pl.ntiles_m - 1) * 64 + wr);
-        const long long it0 = item_at_weight(wtot * blockIdx.x / gridDim.x, pl, wr);
-        const long long it1 = item_at_weight(wtot * (blockIdx.x + 1) / gridDim.x, pl, wr);
-        first = item_at(it0, pl);
+    auto layer_range = [&](int l, ItemPos& first, int& nt) -> int {  // first item, tiles per instance; returns how many items
+        nt = a.ntiles[l];
+        // weight of the last tile of an instance: its 32-column groups out of TMB/32, in 64ths
+        const int last_cols = min(TMB, M + 1 - (nt - 1) * TMB);
+        const int wr = max(1, ((last_cols + 31) / 32) * 64 / (TMB / 32));
+        const long long wtot = (long long)a.nactive[l] * pl.nsb * ((long long)(nt - 1) * 64 + wr);
+        const long long it0 = item_at_weight(wtot * blockIdx.x / gridDim.x, nt, pl.nsb, wr);
+        const long long it1 = item_at_weight(wtot * (blockIdx.x + 1) / gridDim.x, nt, pl.nsb, wr);
+        first = item_at(it0, nt, pl.nsb);
         return (int)(it1 - it0);
     };
 
@@ -339,9 +358,10 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         int n = 0;                                        // chunk counter
         for (int l = l_first; l < l_last; ++l) {
         ItemPos pos;
-        const int nit = layer_range(l, pos);
+        int nt;
+        const int nit = layer_range(l, pos, nt);
         const int row0 = a.C ? (l - 1) * S : ((l - 1) & 1) * a.B * S;      // row of (instance 0, layer l-1, s'=0)
-        for (int q = 0; q < nit; ++q, item_next(pos, pl)) {
+        for (int q = 0; q < nit; ++q, item_next(pos, nt, pl.nsb)) {
             const int i = a.order[pos.oi];
             const int m0 = pos.mt * TMB;
             if (MULTI && tile_done && l > 1) {
@@ -349,9 +369,10 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 const int need = (l - 1) * pl.nsb;
                 // one lane per tile polls (relaxed), then one acquire fence for the warp
                 bool ok = true;
-                for (int t0 = max(0, pos.mt - kdep); t0 <= pos.mt && ok; t0 += 32) {
+                const int tlast = min(pos.mt, a.ntiles[l - 1] - 1);      // tiles the previous layer did not run store nothing
+                for (int t0 = max(0, pos.mt - kdep); t0 <= tlast && ok; t0 += 32) {
                     const int t = t0 + lane;
-                    if (t <= pos.mt) {
+                    if (t <= tlast) {
                         const int32_t* c = tile_done + (size_t)i * pl.ntiles_m + t;
                         int spins = 0;
                         while (ld_relaxed_gpu(c) < need) {
@@ -410,8 +431,9 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         int n = 0;
         for (int l = l_first; l < l_last; ++l) {
         ItemPos pos;
-        const int nit = layer_range(l, pos);
-        for (int q = 0; q < nit; ++q, item_next(pos, pl)) {
+        int nt;
+        const int nit = layer_range(l, pos, nt);
+        for (int q = 0; q < nit; ++q, item_next(pos, nt, pl.nsb)) {
             const int i = a.order[pos.oi];
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);
@@ -482,8 +504,9 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         };
         for (int l = l_first; l < l_last; ++l) {
         ItemPos pos;
-        const int nit = layer_range(l, pos);
-        for (int q = 0; q < nit; ++q, item_next(pos, pl), ++it) {
+        int nt;
+        const int nit = layer_range(l, pos, nt);
+        for (int q = 0; q < nit; ++q, item_next(pos, nt, pl.nsb), ++it) {
             if (!mbar_wait(&out_full, it & 1)) {
                 if (lane == 0) atomicExch(a.err, 1);
                 return;
@@ -546,8 +569,9 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
     int n = 0, it = 0;
     for (int l = l_first; l < l_last; ++l) {
     ItemPos pos;
-    const int nit = layer_range(l, pos);
-    for (int q = 0; q < nit; ++q, item_next(pos, pl), ++it) {
+    int nt;
+    const int nit = layer_range(l, pos, nt);
+    for (int q = 0; q < nit; ++q, item_next(pos, nt, pl.nsb), ++it) {
         const int mw = pos.mt * TMB + ms * (32 * TM);       // first column of this warp
         // 32-column groups of this warp that hold at least one column <= M
         const int nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
@@ -767,6 +791,8 @@ WsLayout galv_ws_layout(const galv_shape* sh)
     w.nactive = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.scratch = off; off = align256(off + (size_t)2 * (sh->Lmax + 2) * 4);
     w.err = off;     off = align256(off + 8);                  // error flag, largest mem
+    w.minmem_l = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
+    w.ntiles = off;   off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.tile_done = off; off = align256(off + (size_t)sh->B * ((sh->M + 128) / 128) * 4);   // per (instance, tile of >= 128 columns)
     w.roll = off;
     if (!(sh->flags & GALV_STORE_C_FULL)) off = align256(off + (size_t)2 * sh->B * sh->S * sh->m_pitch * 4);
@@ -858,8 +884,16 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(a.err, 0, 8, st);
     if (e != cudaSuccess) return e;
-    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1);
-    schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.L, a.status, a.order, a.nactive, a.scratch);
+    const bool reference = (sh->flags & GALV_KERNEL_REFERENCE) != 0;
+    DpPlan pl;
+    std::memset(&pl, 0, sizeof(pl));
+    if (!reference && !galv_dp_make_plan(ctx, sh, &pl)) return cudaErrorInvalidConfiguration;
+    if (reference) { pl.tmb = 256; pl.ntiles_m = (a.M + 256) / 256; }
+    e = cudaMemsetAsync(a.minmem_l, 0x7f, (size_t)(Lmax + 1) * 4, st);
+    if (e != cudaSuccess) return e;
+    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1, a.minmem_l);
+    schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.M, pl.tmb, pl.ntiles_m, a.L, a.status, a.order, a.nactive, a.scratch,
+                                         a.minmem_l, a.ntiles);
     {
         int gx = (a.m_pitch + 255) / 256;
         if (gx > 8) gx = 8;
@@ -877,9 +911,6 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-    const bool reference = (sh->flags & GALV_KERNEL_REFERENCE) != 0;
-    DpPlan pl;
-    if (!reference && !galv_dp_make_plan(ctx, sh, &pl)) return cudaErrorInvalidConfiguration;
     CUtensorMap maps[2];
     std::memset(maps, 0, sizeof(maps));
     if (!reference) {
