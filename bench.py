@@ -37,9 +37,10 @@ METRIC, UNIT = "dp_cell_updates_per_s", "cells/s"
 # Integer-ALU peak of one B200: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min
 # (one min-plus relaxation) per lane per clock.
 ALU_PEAK_GOPS = 148 * 64 * 1.965
-# DRAM bytes (read + write) of one layer_tiled_kernel launch, from the committed ncu captures under
-# profiles/ (a capture launch covers the same units as a benchmark launch: every instance, one layer).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"config3_heterogeneous": 493.9e6, "config4_research_sweep": 501.9e6}
+# DRAM bytes (read + write) per LAYER of the layer_tiled_kernel, from the committed ncu captures under
+# profiles/ (captured on the first layers of the same batch: the kernel's traffic grows in proportion
+# to the layers a launch covers, so a launch over Lmax-1 layers moves (Lmax-1) times this).
+NCU_TRAFFIC_BYTES_PER_LAYER = {"config3_heterogeneous": 528.2e6, "config4_research_sweep": 542.2e6}
 
 
 def workload_for(k: int, rank: int = 0, batch: int = 0, layers: int = 0):
@@ -181,8 +182,9 @@ def time_steps(torch, fn, steps, warmup, barrier):
 
 
 def launches_per_step(w) -> int:
-    # cost + trans kernels, validate + schedule + base layer + (Lmax-1) layer kernels + copy-last + finalize, backtrack
-    return (2 if w.has_model else 0) + 3 + (w.Lmax - 1) + 2 + 1
+    # cost + trans kernels, validate + schedule + base layer, ONE cooperative launch over all layers,
+    # copy-last + finalize, backtrack
+    return (2 if w.has_model else 0) + 3 + 1 + 2 + 1
 
 
 def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):
@@ -251,9 +253,9 @@ def main():
     t = max_over_ranks(r["seconds"])
     clocks = clk.summary()
     value = world * w.cells * args.steps / t
-    layer_s = r["layer_kernel_ms_avg"] * 1e-3
-    relax_per_launch = int((np.minimum(w.L, w.Lmax) - 1).clip(min=0).sum()) * (w.M + 1) * w.S * w.S / max(1, w.Lmax - 1)
-    achieved = relax_per_launch / layer_s / 1e9
+    kernel_s = r["layer_loop_ms"] * 1e-3                     # the one launch that runs every layer
+    relax_per_launch = w.relaxations
+    achieved = relax_per_launch / kernel_s / 1e9
     del sb
     torch.cuda.empty_cache()
 
@@ -284,10 +286,14 @@ def main():
         "searches_per_s": world * w.B * args.steps / t, "relaxations_per_s": world * w.relaxations * args.steps / t,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(w) * args.steps,
         "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_GOPS, "unit": "G add-min/s",
-                     "frac": achieved / ALU_PEAK_GOPS, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
-                     "traffic_unit": "bytes per launch (ncu dram read+write)",
-                     "algorithmic_bytes_per_launch": 2 * 4 * w.B * w.S * w.m_pitch,
-                     "kernel": "layer_tiled_kernel", "launch_ms": r["layer_kernel_ms_avg"],
+                     "frac": achieved / ALU_PEAK_GOPS,
+                     "traffic": (NCU_TRAFFIC_BYTES_PER_LAYER[w.name] * (w.Lmax - 1)
+                                 if w.name in NCU_TRAFFIC_BYTES_PER_LAYER else None),
+                     "traffic_unit": "bytes per launch (ncu dram read+write per layer x layers)",
+                     "algorithmic_bytes_per_launch": 2 * 4 * w.B * w.S * w.m_pitch * (w.Lmax - 1),
+                     "algorithmic_ops_per_launch": relax_per_launch,
+                     "kernel": "layer_tiled_kernel (one cooperative launch over all layers)",
+                     "launch_ms": r["layer_loop_ms"],
                      "peak_source": "derived: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min per lane per clock"},
     }
 
