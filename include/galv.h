@@ -231,6 +231,37 @@ int galv_compact_tables(galv_ctx* ctx, const galv_shape* shape, int32_t S_kept, 
 /* Turn a plan over kept strategies back into original indices, in place: plan[e] = map[plan[e]] where >= 0. */
 int galv_expand_plan(galv_ctx* ctx, int32_t B, int32_t Lmax, const int32_t* map, int32_t* plan, void* stream);
 
+/*
+ * Cost and memory of GIVEN plans under the current tables (Sections 3-4: when the selector
+ * re-evaluates during training it weighs the running plan against the new optimum):
+ * cost[i] = sum_l time(l,p_l) + sum_{l>=1} trans(p_{l-1},p_l), mem_total[i] = sum_l mem(l,p_l)
+ * over the L[i] layers of instance i, as int64; both -1 when L[i] is out of range or the plan
+ * has an entry outside 0..S-1 among those layers.  plan int32 [B][Lmax].  All device pointers.
+ */
+int galv_plan_cost(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                   const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,
+                   const int32_t* plan, int64_t* cost, int64_t* mem_total, void* stream);
+
+/*
+ * Re-search pipeline (Sections 3-4: the selector re-runs at intervals from fresh measurements).
+ * galv_graph_create captures galv_eval_costs (when layers != NULL) -> galv_dp_search ->
+ * galv_backtrack on the given device buffers into a CUDA graph; galv_graph_launch replays it on
+ * a stream.  Between replays the caller may overwrite the CONTENTS of any input buffer (typically
+ * inst: measured FLOP rate, link bandwidth, micro-batch); pointers and shape are frozen.
+ * Arguments are those of the three calls; `stream` must be a non-default stream that is not
+ * capturing; the galv_graph holds no device memory.  One replay in flight at a time.
+ */
+typedef struct galv_graph galv_graph;
+int galv_graph_create(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                      const galv_layer_desc* layers, int64_t layer_stride_B,
+                      const galv_strategy_desc* strat, const galv_inst_params* inst,
+                      int32_t* time_q, int32_t* mem_q, int32_t* trans_q,
+                      int32_t* C, uint8_t* A, int32_t* C_last, void* workspace, size_t workspace_bytes,
+                      const int32_t* budget, int32_t* opt_cost, int32_t* plan, int32_t* mem_used,
+                      int32_t* status, void* stream, galv_graph** out);
+int galv_graph_launch(galv_ctx* ctx, galv_graph* graph, void* stream);
+int galv_graph_destroy(galv_graph* graph);
+
 /* Bytes of device arena galv_search_host needs (0 on invalid shape). */
 size_t galv_search_host_arena_bytes(const galv_ctx* ctx, const galv_shape* shape, int with_model);
 

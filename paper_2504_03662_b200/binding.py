@@ -24,7 +24,8 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgalv.so"
 EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "galv_eval_costs",
            "galv_dp_workspace_bytes", "galv_dp_search", "galv_backtrack", "galv_search_host_arena_bytes",
            "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_dp_search_static", "galv_select_best", "galv_prune_strategies",
-           "galv_compact_tables", "galv_expand_plan")
+           "galv_compact_tables", "galv_expand_plan", "galv_plan_cost", "galv_graph_create", "galv_graph_launch",
+           "galv_graph_destroy")
 
 
 class galv_shape(C.Structure):
@@ -67,6 +68,10 @@ def load_library() -> C.CDLL:
     lib.galv_prune_strategies.argtypes = [vp, shp] + [vp] * 8
     lib.galv_compact_tables.argtypes = [vp, shp, C.c_int32] + [vp] * 8
     lib.galv_expand_plan.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, vp]
+    lib.galv_plan_cost.argtypes = [vp, shp] + [vp] * 8
+    lib.galv_graph_create.argtypes = [vp, shp, vp, vp, i64, vp, vp] + [vp] * 7 + [sz] + [vp] * 6 + [C.POINTER(vp)]
+    lib.galv_graph_launch.argtypes = [vp, vp, vp]
+    lib.galv_graph_destroy.argtypes = [vp]
     lib.galv_search_host_arena_bytes.argtypes = [vp, shp, C.c_int]
     lib.galv_search_host_arena_bytes.restype = sz
     lib.galv_search_host.argtypes = [vp, shp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -154,6 +159,26 @@ class Galv:
 
     def galv_expand_plan(self, B, Lmax, map_, plan):
         self._check(self.lib.galv_expand_plan(self.h, B, Lmax, _ptr(map_), _ptr(plan), _stream()))
+
+    def galv_plan_cost(self, shape, L, time_q, mem_q, trans_q, plan, cost, mem_total):
+        self._check(self.lib.galv_plan_cost(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),
+                                            _ptr(plan), _ptr(cost), _ptr(mem_total), _stream()))
+
+    def galv_graph_create(self, shape, L, layers, layer_stride_B, strat, inst, time_q, mem_q, trans_q, Ct, At, C_last,
+                          workspace, budget, opt_cost, plan, mem_used, status, stream: int):
+        g = C.c_void_p()
+        self._check(self.lib.galv_graph_create(self.h, C.byref(shape), _ptr(L), _ptr(layers), layer_stride_B, _ptr(strat),
+                                               _ptr(inst), _ptr(time_q), _ptr(mem_q), _ptr(trans_q), _ptr(Ct), _ptr(At),
+                                               _ptr(C_last), _ptr(workspace),
+                                               workspace.numel() * workspace.element_size(), _ptr(budget), _ptr(opt_cost),
+                                               _ptr(plan), _ptr(mem_used), _ptr(status), stream, C.byref(g)))
+        return g
+
+    def galv_graph_launch(self, graph, stream: Optional[int] = None):
+        self._check(self.lib.galv_graph_launch(self.h, graph, _stream() if stream is None else stream))
+
+    def galv_graph_destroy(self, graph):
+        self.lib.galv_graph_destroy(graph)
 
     def galv_backtrack(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, budget, opt_cost, plan, mem_used, status):
         self._check(self.lib.galv_backtrack(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),
