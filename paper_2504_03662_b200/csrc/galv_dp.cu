@@ -10,12 +10,16 @@
 // CUDA-core GEMM: an item is (instance, tile of m', block of s); warps own a
 // register tile of (TM x 32 columns) x (8 strategies); the previous layer's rows
 // and the matching rows of the S x S transition matrix are staged in shared memory
-// by bulk async copies (TMA unit) issued by a producer warp, in a multi-stage
-// mbarrier pipeline over chunks of s'.  One fused add-min instruction per
+// by tensor-map TMA loads issued by a producer warp, in a multi-stage mbarrier
+// pipeline over chunks of s'; the outputs leave through a staging tile and TMA
+// bulk stores issued by a store warp.  One fused add-min instruction per
 // relaxation; no tensor cores (min-plus is not a multiply-add contraction).
 //
-// One launch per layer (a layer needs all of the previous one); launches are
-// plain stream work, so a caller may capture the whole search in a CUDA graph.
+// A layer needs the previous one.  With the full table kept, all layers run in one
+// cooperative launch: CTAs publish finished tiles in global counters and start a
+// tile of the next layer as soon as the tiles it reads are published (bounded
+// waits).  With an argmin table or the two-layer rolling buffer: one launch per
+// layer.  Either way plain stream work, capturable in a CUDA graph.
 
 #include <cuda.h>
 
@@ -250,8 +254,9 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 //       stage, runs one fused add-min per relaxation, releases the stage, and after the last
 //       chunk adds time(l,s) and writes its tile into the staging tile, row s shifted by
 //       mem(l,s) mod 4 so that column m' + mem(l,s) of the table is 16-byte aligned with it.
-// Stages are handed over with mbarriers (full: bytes landed and record written; empty: every consumer warp done),
-// so there is no block-wide barrier in the loop.  Every wait is bounded.
+// Stages are handed over with mbarriers (full: bytes landed and record written; empty: every consumer
+// warp done; out_full / out_empty for the staging tile), so there is no block-wide barrier in the
+// loop.  Every wait is bounded; a wait that runs out sets the error flag and the role returns.
 
 constexpr int kMaxStages = 4;
 
