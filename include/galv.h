@@ -61,6 +61,9 @@ extern "C" {
 #define GALV_STORE_ARGMIN 2 /* write the argmin table A */
 #define GALV_KERNEL_REFERENCE 256 /* run the recurrence with the simple one-thread-per-cell kernel (slow; cross-checks) */
 #define GALV_KERNEL_PER_LAYER 512 /* one launch per layer instead of one cooperative launch over all layers */
+#define GALV_SKIP_INFEASIBLE 1024 /* tiles wholly below the previous layer's feasibility frontier (sum of the
+                                     layers' smallest mem) read only +inf: write their +inf results without
+                                     loading or relaxing anything.  Same tables, less work on tight budgets. */
 
 typedef struct galv_ctx galv_ctx;
 

@@ -193,6 +193,7 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const 
     a.maxmem = a.err + 1;
     a.minmem_l = reinterpret_cast<int32_t*>(ws + w.minmem_l);
     a.ntiles = reinterpret_cast<int32_t*>(ws + w.ntiles);
+    a.front = reinterpret_cast<int32_t*>(ws + w.front);
     a.status = status;
     cudaError_t e = galv_dp_launch(ctx, sh, a, (cudaStream_t)stream);
     return e == cudaSuccess ? GALV_OK : cuda_fail(ctx, "galv_dp_search", e);

@@ -98,7 +98,7 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 __global__ void validate_kernel(int B, int Lmax, int S, int M, const int32_t* __restrict__ L,
                                 const int32_t* __restrict__ time_q, const int32_t* __restrict__ mem_q,
                                 const int32_t* __restrict__ trans_q, int32_t* __restrict__ status,
-                                int32_t* __restrict__ maxmem, int32_t* __restrict__ minmem_l)
+                                int32_t* __restrict__ maxmem, int32_t* __restrict__ minmem_l, int32_t* __restrict__ front)
 {
     const int i = blockIdx.x;
     __shared__ long long s_sum;
@@ -145,12 +145,25 @@ __global__ void validate_kernel(int B, int Lmax, int S, int M, const int32_t* __
         s_bad = st;
     }
     __syncthreads();
-    if (s_bad == 0)
+    if (s_bad == 0) {
         for (int l = threadIdx.x; l < Li; l += blockDim.x) {      // smallest mem of each layer over the valid instances
             int mn = 0x7fffffff;
             for (int s = 0; s < S; ++s) mn = min(mn, mq[l * S + s]);
             atomicMin(&minmem_l[l], mn);
+            if (front) front[(size_t)i * Lmax + l] = mn;
         }
+        if (front) {
+            // feasibility frontier: no cell of layer l is finite below the sum of the layers' smallest mem
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                long long run = 0;
+                for (int l = 0; l < Li; ++l) {
+                    run += front[(size_t)i * Lmax + l];
+                    front[(size_t)i * Lmax + l] = (int32_t)min(run, (long long)M + 1);
+                }
+            }
+        }
+    }
 }
 
 // Single CTA: nactive[l] = valid instances with L > l; order = valid instances, longest first.
@@ -399,11 +412,18 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
             const int yc = row0 + i * inst_rows;
             const int32_t* T = a.trans_q + (size_t)i * S * S + sb0;
+            // a tile wholly below the previous layer's feasibility frontier reads nothing but +inf: no loads
+            const bool skip = a.front && m0 + TMB - 1 < a.front[(size_t)i * a.Lmax + (l - 1)];
             for (int kc = 0; kc < NKC; ++kc, ++n) {
                 const int st = n % NST;
                 if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
+                }
+                if (skip) {
+                    if (lane == 0) mbar_arrive(&full_bar[st]);
+                    __syncwarp();
+                    continue;
                 }
                 const int k0 = kc * KS;
                 int32_t* cs = stage0 + st * stage_elems;
@@ -443,6 +463,7 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);
             const size_t qrow = ((size_t)i * a.Lmax + l) * S + sb0;
+            const int skip = a.front && pos.mt * TMB + TMB - 1 < a.front[(size_t)i * a.Lmax + (l - 1)];
             // this s-block's mem and time row, two strategies per lane (SB <= 64)
             const int mq0 = lane < sbw ? __ldg(a.mem_q + qrow + lane) : 0;
             const int mq1 = lane + 32 < sbw ? __ldg(a.mem_q + qrow + lane + 32) : 0;
@@ -454,13 +475,14 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
+                int32_t* meta = meta0 + st * META;
                 if (kc == NKC - 1) {
-                    int32_t* meta = meta0 + st * META;
                     if (lane < SB) { meta[lane] = mq0; meta[SB + lane] = tq0; }
                     if (lane + 32 < SB) { meta[lane + 32] = mq1; meta[SB + lane + 32] = tq1; }
                     if (lane == 0) meta[2 * SB] = i;
-                    __syncwarp();
                 }
+                if (lane == 0) meta[2 * SB + 1] = skip;           // the consumers leave this chunk's k-steps out
+                __syncwarp();
                 if (lane == 0) mbar_arrive(&full_bar[st]);
             }
             if (pos.mt == 0) {
@@ -595,7 +617,8 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 return;
             }
             const int k0 = kc * KS;
-            const int kn = min(KS, S - k0);
+            // nothing but +inf to read (see the producer): the accumulators stay at +inf
+            const int kn = meta0[st * META + 2 * SB + 1] ? 0 : min(KS, S - k0);
             // this warp's columns inside their box, and its 8 trans columns
             const int32_t* cs = stage0 + st * stage_elems + ((ms * (32 * TM)) / BOXC) * (KS * BOXC) + (ms * (32 * TM)) % BOXC + lane;
             const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
@@ -798,6 +821,7 @@ WsLayout galv_ws_layout(const galv_shape* sh)
     w.err = off;     off = align256(off + 8);                  // error flag, largest mem
     w.minmem_l = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.ntiles = off;   off = align256(off + (size_t)(sh->Lmax + 1) * 4);
+    w.front = off;    off = align256(off + (size_t)sh->B * sh->Lmax * 4);
     w.tile_done = off; off = align256(off + (size_t)sh->B * ((sh->M + 128) / 128) * 4);   // per (instance, tile of >= 128 columns)
     w.roll = off;
     if (!(sh->flags & GALV_STORE_C_FULL)) off = align256(off + (size_t)2 * sh->B * sh->S * sh->m_pitch * 4);
@@ -896,7 +920,8 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     if (reference) { pl.tmb = 256; pl.ntiles_m = (a.M + 256) / 256; }
     e = cudaMemsetAsync(a.minmem_l, 0x7f, (size_t)(Lmax + 1) * 4, st);
     if (e != cudaSuccess) return e;
-    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1, a.minmem_l);
+    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1, a.minmem_l,
+                                       (sh->flags & GALV_SKIP_INFEASIBLE) ? a.front : nullptr);
     schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.M, pl.tmb, pl.ntiles_m, a.L, a.status, a.order, a.nactive, a.scratch,
                                          a.minmem_l, a.ntiles);
     {
@@ -931,6 +956,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     // (with the two-layer rolling buffer a layer would overwrite cells a slower CTA still reads)
     const bool persistent = !reference && a.C && !a.A && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
     DpArgs ap = a;
+    if (!(sh->flags & GALV_SKIP_INFEASIBLE)) ap.front = nullptr;
     ap.tile_done = nullptr;
     ap.maxmem = a.err + 1;
     if (persistent) {

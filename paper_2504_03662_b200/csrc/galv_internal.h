@@ -52,6 +52,7 @@ struct DpArgs {
     int32_t* tile_done;  // [B][ntiles_m] finished items per (instance, tile); NULL when layers are separate launches
     int32_t* maxmem;     // largest mem over the valid instances (min(.., M+1))
     int32_t* minmem_l;   // [Lmax+1] smallest mem of each layer over the valid instances
+    int32_t* front;      // [B][Lmax] feasibility frontier (sum of the layers' smallest mem), or NULL when tiles are never skipped
     int32_t* ntiles;     // [Lmax+1] tiles per instance that can store anything in layer l
     int32_t* status;
 };
@@ -60,7 +61,7 @@ struct DpArgs {
 int galv_set_error(galv_ctx* ctx, int code, const char* text);
 
 // workspace carve-up (offsets in bytes, all 256-aligned)
-struct WsLayout { size_t order, nactive, scratch, err, minmem_l, ntiles, tile_done, roll, total; };
+struct WsLayout { size_t order, nactive, scratch, err, minmem_l, ntiles, front, tile_done, roll, total; };
 WsLayout galv_ws_layout(const galv_shape* sh);
 
 bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* plan);

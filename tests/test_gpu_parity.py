@@ -122,7 +122,7 @@ SHAPES = [  # B, Lmax, S, M, kwargs
 ]
 
 
-@pytest.mark.parametrize("flags", [1, 3, 2, 1 | 512])
+@pytest.mark.parametrize("flags", [1, 3, 2, 1 | 512, 1 | 1024, 2 | 1024])
 @pytest.mark.parametrize("k", range(len(SHAPES)))
 def test_random_shapes(orc, galv, flags, k):
     B, Lmax, S, M, kw = SHAPES[k]
@@ -194,11 +194,12 @@ def test_config4_full_size(orc, galv):
     assert (res2["opt_cost"] == res["opt_cost"]).all() and (res2["plan"] == res["plan"]).all()
 
 
-def test_config3_full_size(orc, galv):
+@pytest.mark.parametrize("flags", [1, 1 | 1024])      # plain; tiles below the feasibility frontier skipped
+def test_config3_full_size(orc, galv, flags):
     import torch
     w = inputs.config3()
     idx = [0, 37, 127]
-    sb, res = check_batch(orc, galv, w, 1, idx=idx)
+    sb, res = check_batch(orc, galv, w, flags, idx=idx)
     assert (res["status"] == 0).all()
     tq, mq, xq = oracle_tables(orc, w)
     _properties_all(orc, w, tq, mq, xq, sb, res)
