@@ -61,6 +61,9 @@ extern "C" {
 #define GALV_STORE_ARGMIN 2 /* write the argmin table A */
 #define GALV_KERNEL_REFERENCE 256 /* run the recurrence with the simple one-thread-per-cell kernel (slow; cross-checks) */
 #define GALV_KERNEL_PER_LAYER 512 /* one launch per layer instead of one cooperative launch over all layers */
+#define GALV_DEBUG_WITHHOLD_LOAD 2048 /* test hook for the time-out path: one CTA never receives its first stage, every
+                                         bounded wait that depends on it runs out (about a second each), status gets
+                                         GALV_STATUS_TIMEOUT and the call's results are void; nothing faults or hangs */
 #define GALV_SKIP_INFEASIBLE 1024 /* tiles wholly below the previous layer's feasibility frontier (sum of the
                                      layers' smallest mem) read only +inf: write their +inf results without
                                      loading or relaxing anything.  Same tables, less work on tight budgets. */

@@ -195,6 +195,7 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const 
     a.ntiles = reinterpret_cast<int32_t*>(ws + w.ntiles);
     a.front = reinterpret_cast<int32_t*>(ws + w.front);
     a.status = status;
+    a.withhold = 0;
     cudaError_t e = galv_dp_launch(ctx, sh, a, (cudaStream_t)stream);
     return e == cudaSuccess ? GALV_OK : cuda_fail(ctx, "galv_dp_search", e);
 }

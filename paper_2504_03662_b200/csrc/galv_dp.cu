@@ -31,7 +31,22 @@ namespace {
 
 constexpr int kInf = GALV_INF;
 constexpr int TS = 8;                 // strategies per warp register tile
-constexpr int kSpinLimit = 1 << 22;   // bounded mbarrier polling (each poll may block for a while in hardware)
+// Every device-side wait gives up after about a second (SM clock cycles; checked every few polls):
+// the role sets the error flag and returns, the host sees GALV_STATUS_TIMEOUT, the context stays usable.
+constexpr long long kWaitLimitCycles = 2000000000LL;
+
+struct WaitClock {
+    long long t0;
+    int polls;
+    __device__ WaitClock() : t0(0), polls(0) {}
+    // true when the limit ran out
+    __device__ bool expired() {
+        if ((++polls & 255) != 0) return false;
+        const long long now = clock64();
+        if (t0 == 0) { t0 = now; return false; }
+        return now - t0 > kWaitLimitCycles;
+    }
+};
 
 // ---------------------------------------------------------------- PTX helpers
 
@@ -81,9 +96,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait: false when the limit ran out.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    for (int i = 0; i < kSpinLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
+    WaitClock wc;
+    while (!mbar_try_wait(bar, parity))
+        if (wc.expired()) return false;
+    return true;
 }
 // 1-D bulk async copy global -> shared, completion counted in bytes on an mbarrier.
 // dst, src 16-byte aligned, bytes a multiple of 16.
@@ -392,9 +408,9 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                     const int t = t0 + lane;
                     if (t <= tlast) {
                         const int32_t* c = tile_done + (size_t)i * pl.ntiles_m + t;
-                        int spins = 0;
+                        WaitClock wc;
                         while (ld_relaxed_gpu(c) < need) {
-                            if (++spins > kSpinLimit) { ok = false; break; }
+                            if (wc.expired()) { ok = false; break; }
                             __nanosleep(64);
                         }
                     }
@@ -425,6 +441,7 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                     __syncwarp();
                     continue;
                 }
+                if (a.withhold && blockIdx.x == 0 && n == 0) continue;   // test hook: a stage that never fills
                 const int k0 = kc * KS;
                 int32_t* cs = stage0 + st * stage_elems;
                 int32_t* ts = cs + KS * TMB;
@@ -569,9 +586,9 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 int32_t* mine = tile_done + (size_t)i * pl.ntiles_m + pos.mt;
                 if (pos.mt == 0) {                                // the helper's fill of this tile (it runs ahead)
                     ++nfill;
-                    int spins = 0;
+                    WaitClock wc;
                     while (*reinterpret_cast<volatile int*>(&fill_count) < nfill) {
-                        if (++spins > kSpinLimit) {
+                        if (wc.expired()) {
                             if (lane == 0) atomicExch(a.err, 1);
                             return;
                         }
@@ -956,6 +973,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     // (with the two-layer rolling buffer a layer would overwrite cells a slower CTA still reads)
     const bool persistent = !reference && a.C && !a.A && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
     DpArgs ap = a;
+    ap.withhold = (sh->flags & GALV_DEBUG_WITHHOLD_LOAD) != 0;
     if (!(sh->flags & GALV_SKIP_INFEASIBLE)) ap.front = nullptr;
     ap.tile_done = nullptr;
     ap.maxmem = a.err + 1;

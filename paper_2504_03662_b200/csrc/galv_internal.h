@@ -55,6 +55,7 @@ struct DpArgs {
     int32_t* front;      // [B][Lmax] feasibility frontier (sum of the layers' smallest mem), or NULL when tiles are never skipped
     int32_t* ntiles;     // [Lmax+1] tiles per instance that can store anything in layer l
     int32_t* status;
+    int withhold;        // test hook: CTA 0 never loads its first chunk, so that the bounded waits run out
 };
 
 // records `text` as the context's last error and returns `code`

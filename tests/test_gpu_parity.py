@@ -291,3 +291,21 @@ def test_boundary_errors(galv):
 def test_alu_probe_runs(galv):
     rates = [galv.galv_probe_int_alu(k, 512) for k in (0, 1, 2)]
     assert all(1e11 < r < 1e15 for r in rates), rates
+
+
+@pytest.mark.parametrize("flags", [1, 1 | 512])
+def test_bounded_waits_run_out_cleanly(orc, galv, flags):
+    """A stage that never fills: the waits give up, the status says TIMEOUT, the context keeps working."""
+    import time
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    w = inputs.random_tables(3, 4, 5, 12, 300, mem_lo=1, mem_hi=60)
+    bad = SearchBuffers(galv, w, flags | gb.DEBUG_WITHHOLD_LOAD)
+    t0 = time.time()
+    bad.dp_search()
+    torch.cuda.synchronize()                               # returns: no hang, no fault
+    assert time.time() - t0 < 60
+    assert (bad.status.cpu().numpy() & gb.STATUS_TIMEOUT).all()
+    # the same context and device then search normally
+    check_batch(orc, galv, w, flags)
