@@ -59,6 +59,8 @@ extern "C" {
 /* shape.flags */
 #define GALV_STORE_C_FULL 1 /* keep every layer of C (needed to backtrack without A) */
 #define GALV_STORE_ARGMIN 2 /* write the argmin table A */
+#define GALV_TRANS_PER_LAYER 4 /* trans_q is [B][Lmax][S][S]: matrix l is paid between layers l-1 and l (matrix 0 unused);
+                                  for galv_dp_search, galv_backtrack, galv_plan_cost, galv_search_host, galv_graph_create */
 #define GALV_KERNEL_REFERENCE 256 /* run the recurrence with the simple one-thread-per-cell kernel (slow; cross-checks) */
 #define GALV_KERNEL_PER_LAYER 512 /* one launch per layer instead of one cooperative launch over all layers */
 #define GALV_DEBUG_WITHHOLD_LOAD 2048 /* test hook for the time-out path: one CTA never receives its first stage, every

@@ -26,6 +26,9 @@
  * 0..M inclusive.  +inf is ORC_INF = 2^30-1, absorbing.
  *
  * Layout here is the recurrence's own index order, C[l][m][s] with s fastest.
+ * trans is one S x S matrix, or one per layer: tl is the number of entries between
+ * the matrices of consecutive layers (0: one matrix; S*S: matrix l is paid between
+ * layers l-1 and l, matrix 0 is unused).
  *
  * Parity pins (tests, CPU only): brute force on tiny shapes, monotonicity in m,
  * hand-derived worked example, S=1 closed form, trans=0 multiple-choice
@@ -46,7 +49,7 @@ enum { ORC_INFEASIBLE = 1, ORC_BAD_INPUT = 2, ORC_OVERFLOW_RISK = 4 };
 
 /* Input check: entries non-negative, and no finite path sum can reach ORC_INF:
  * sum_l max_s time(l,s) + (L-1) * max trans < ORC_INF. */
-int orc_validate(int L, int S, const int32_t *time, const int32_t *mem, const int32_t *trans)
+int orc_validate(int L, int S, const int32_t *time, const int32_t *mem, const int32_t *trans, int64_t tl)
 {
     int st = 0;
     int64_t sum = 0, tmax = 0;
@@ -59,17 +62,18 @@ int orc_validate(int L, int S, const int32_t *time, const int32_t *mem, const in
         }
         sum += mx;
     }
-    for (int k = 0; k < S * S; k++) {
-        if (trans[k] < 0) st |= ORC_BAD_INPUT;
-        if (trans[k] > tmax) tmax = trans[k];
-    }
+    for (int l = (tl ? 1 : 0); l < (tl ? L : 1); l++)
+        for (int k = 0; k < S * S; k++) {
+            if (trans[l * tl + k] < 0) st |= ORC_BAD_INPUT;
+            if (trans[l * tl + k] > tmax) tmax = trans[l * tl + k];
+        }
     if (!(st & ORC_BAD_INPUT) && sum + (int64_t)(L - 1) * tmax >= ORC_INF) st |= ORC_OVERFLOW_RISK;
     return st;
 }
 
 /* The recurrence.  C and A are [L][M+1][S]; A may be NULL.  A holds the lowest
  * minimising s' (255 where the cell is +inf and on layer 0). */
-void orc_dp(int L, int S, int M, const int32_t *time, const int32_t *mem, const int32_t *trans,
+void orc_dp(int L, int S, int M, const int32_t *time, const int32_t *mem, const int32_t *trans, int64_t tl,
             int32_t *C, uint8_t *A)
 {
     const int64_t W = (int64_t)(M + 1) * S;
@@ -88,7 +92,7 @@ void orc_dp(int L, int S, int M, const int32_t *time, const int32_t *mem, const 
                     const int32_t *prev = C + (l - 1) * W + mp * S;
                     for (int sp = 0; sp < S; sp++)
                         if (prev[sp] < ORC_INF) {
-                            int64_t v = (int64_t)prev[sp] + trans[sp * S + s];
+                            int64_t v = (int64_t)prev[sp] + trans[l * tl + sp * S + s];
                             if (v < best) { best = v; arg = sp; }
                         }
                 }
@@ -101,7 +105,7 @@ void orc_dp(int L, int S, int M, const int32_t *time, const int32_t *mem, const 
  * the walk reads the stored argmin, without it the argmin is found again from
  * C (lowest s' whose candidate equals the cell's pre-time value).
  * Returns status bits; plan[l] = -1 everywhere when infeasible. */
-int orc_backtrack(int L, int S, int M, const int32_t *time, const int32_t *mem, const int32_t *trans,
+int orc_backtrack(int L, int S, int M, const int32_t *time, const int32_t *mem, const int32_t *trans, int64_t tl,
                   const int32_t *C, const uint8_t *A, int budget,
                   int32_t *opt_cost, int32_t *plan, int32_t *mem_used)
 {
@@ -129,7 +133,7 @@ int orc_backtrack(int L, int S, int M, const int32_t *time, const int32_t *mem, 
             int64_t target = (int64_t)C[l * W + m * S + s] - time[l * S + s];
             for (int sp = 0; sp < S; sp++) {
                 int32_t c = C[(l - 1) * W + mp * S + sp];
-                if (c < ORC_INF && (int64_t)c + trans[sp * S + s] == target) { prev_s = sp; break; }
+                if (c < ORC_INF && (int64_t)c + trans[l * tl + sp * S + s] == target) { prev_s = sp; break; }
             }
         }
         m = mp;
@@ -140,14 +144,14 @@ int orc_backtrack(int L, int S, int M, const int32_t *time, const int32_t *mem, 
 }
 
 /* cost(p) and memory of one plan, straight from the definition. */
-void orc_plan_cost(int L, int S, const int32_t *time, const int32_t *mem, const int32_t *trans,
+void orc_plan_cost(int L, int S, const int32_t *time, const int32_t *mem, const int32_t *trans, int64_t tl,
                    const int32_t *plan, int64_t *cost, int64_t *mem_total)
 {
     int64_t c = 0, u = 0;
     for (int l = 0; l < L; l++) {
         c += time[l * S + plan[l]];
         u += mem[l * S + plan[l]];
-        if (l >= 1) c += trans[plan[l - 1] * S + plan[l]];
+        if (l >= 1) c += trans[l * tl + plan[l - 1] * S + plan[l]];
     }
     *cost = c;
     *mem_total = u;
@@ -158,14 +162,14 @@ void orc_plan_cost(int L, int S, const int32_t *time, const int32_t *mem, const 
  * and "strictly better" keeps the first, i.e. the smallest in that order.
  * Returns the number of feasible plans; opt_cost = ORC_INF and plan = -1 if none. */
 int64_t orc_brute_force(int L, int S, int budget, const int32_t *time, const int32_t *mem,
-                        const int32_t *trans, int32_t *opt_cost, int32_t *plan, int32_t *mem_used)
+                        const int32_t *trans, int64_t tl, int32_t *opt_cost, int32_t *plan, int32_t *mem_used)
 {
     int32_t *p = (int32_t *)calloc((size_t)L, sizeof(int32_t));
     int64_t best = -1, best_mem = 0, feasible = 0;
     for (int l = 0; l < L; l++) plan[l] = -1;
     for (;;) {
         int64_t c, u;
-        orc_plan_cost(L, S, time, mem, trans, p, &c, &u);
+        orc_plan_cost(L, S, time, mem, trans, tl, p, &c, &u);
         if (u <= budget) {
             feasible++;
             if (best < 0 || c < best) {

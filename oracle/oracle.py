@@ -51,10 +51,16 @@ def _i32(a):
     return a, a.ctypes.data_as(C.c_void_p)
 
 
+def _tl(trans, L, S):
+    """Layer stride of trans: 0 for one [S][S] matrix, S*S for one matrix per layer ([L][S][S])."""
+    assert trans.shape in ((S, S), (L, S, S)), trans.shape
+    return C.c_int64(0 if trans.ndim == 2 else S * S)
+
+
 def validate(time, mem, trans) -> int:
     time, pt = _i32(time); mem, pm = _i32(mem); trans, px = _i32(trans)
     L, S = time.shape
-    return lib().orc_validate(L, S, pt, pm, px)
+    return lib().orc_validate(L, S, pt, pm, px, _tl(trans, L, S))
 
 
 def dp(time, mem, trans, M: int, want_A: bool = True):
@@ -63,7 +69,7 @@ def dp(time, mem, trans, M: int, want_A: bool = True):
     L, S = time.shape
     Ct = np.empty((L, M + 1, S), np.int32)
     At = np.empty((L, M + 1, S), np.uint8) if want_A else None
-    lib().orc_dp(L, S, M, pt, pm, px, Ct.ctypes.data_as(C.c_void_p),
+    lib().orc_dp(L, S, M, pt, pm, px, _tl(trans, L, S), Ct.ctypes.data_as(C.c_void_p),
                  At.ctypes.data_as(C.c_void_p) if want_A else None)
     return Ct, At
 
@@ -76,7 +82,7 @@ def backtrack(time, mem, trans, Ct, At, budget: int):
     assert 0 <= budget <= M and Ct.flags.c_contiguous
     opt = C.c_int32(); used = C.c_int32()
     plan = np.empty(L, np.int32)
-    st = lib().orc_backtrack(L, S, M, pt, pm, px, Ct.ctypes.data_as(C.c_void_p),
+    st = lib().orc_backtrack(L, S, M, pt, pm, px, _tl(trans, L, S), Ct.ctypes.data_as(C.c_void_p),
                              At.ctypes.data_as(C.c_void_p) if At is not None else None,
                              int(budget), C.byref(opt), plan.ctypes.data_as(C.c_void_p), C.byref(used))
     return opt.value, plan, used.value, st
@@ -88,7 +94,7 @@ def brute_force(time, mem, trans, budget: int):
     L, S = time.shape
     opt = C.c_int32(); used = C.c_int32()
     plan = np.empty(L, np.int32)
-    n = lib().orc_brute_force(L, S, int(budget), pt, pm, px, C.byref(opt),
+    n = lib().orc_brute_force(L, S, int(budget), pt, pm, px, _tl(trans, L, S), C.byref(opt),
                               plan.ctypes.data_as(C.c_void_p), C.byref(used))
     return opt.value, plan, used.value, n
 
@@ -97,7 +103,7 @@ def plan_cost(time, mem, trans, plan):
     time, pt = _i32(time); mem, pm = _i32(mem); trans, px = _i32(trans); plan, pp = _i32(plan)
     L, S = time.shape
     c = C.c_int64(); u = C.c_int64()
-    lib().orc_plan_cost(L, S, pt, pm, px, pp, C.byref(c), C.byref(u))
+    lib().orc_plan_cost(L, S, pt, pm, px, _tl(trans, L, S), pp, C.byref(c), C.byref(u))
     return c.value, u.value
 
 

@@ -46,7 +46,7 @@ Arena arena_layout(const galv_shape* sh, bool with_model)
     a.inst = take(with_model ? B * sizeof(galv_inst_params) : 0);
     a.time_q = take(B * Lm * S * 4);
     a.mem_q = take(B * Lm * S * 4);
-    a.trans_q = take(B * S * S * 4);
+    a.trans_q = take(B * S * S * 4 * ((sh->flags & GALV_TRANS_PER_LAYER) ? Lm : 1));
     a.C = take((sh->flags & GALV_STORE_C_FULL) ? B * Lm * S * P * 4 : 0);
     a.A = take((sh->flags & GALV_STORE_ARGMIN) ? B * Lm * S * P : 0);
     a.C_last = take(B * S * P * 4);
@@ -143,6 +143,10 @@ int galv_eval_costs(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const
         set_err(ctx, "galv_eval_costs: layer_stride_B must be 0 or >= Lmax");
         return GALV_ERR_INVALID_ARG;
     }
+    if (sh->flags & GALV_TRANS_PER_LAYER) {
+        set_err(ctx, "galv_eval_costs: the cost model writes one transition matrix per instance (no GALV_TRANS_PER_LAYER)");
+        return GALV_ERR_INVALID_ARG;
+    }
     cudaError_t e = galv_costs_launch(sh, L, layers, layer_stride_B, strat, inst, time_s, mem_bytes, time_q, mem_q,
                                       trans_q, status, (cudaStream_t)stream);
     return e == cudaSuccess ? GALV_OK : cuda_fail(ctx, "galv_eval_costs", e);
@@ -183,6 +187,7 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const 
     DpArgs a;
     a.B = sh->B; a.Lmax = sh->Lmax; a.S = sh->S; a.M = sh->M; a.m_pitch = sh->m_pitch;
     a.L = L; a.time_q = time_q; a.mem_q = mem_q; a.trans_q = trans_q;
+    a.trans_inst = galv_trans_inst(sh); a.trans_layer = galv_trans_layer(sh);
     a.C = C; a.A = A; a.C_last = C_last;
     a.roll = reinterpret_cast<int32_t*>(ws + w.roll);
     a.order = reinterpret_cast<int32_t*>(ws + w.order);
@@ -281,7 +286,7 @@ int galv_search_host(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, cons
     } else {
         GALV_H2D(ar.time_q, time_q, B * Lm * S * 4);
         GALV_H2D(ar.mem_q, mem_q, B * Lm * S * 4);
-        GALV_H2D(ar.trans_q, trans_q, B * S * S * 4);
+        GALV_H2D(ar.trans_q, trans_q, B * S * S * 4 * ((sh->flags & GALV_TRANS_PER_LAYER) ? Lm : 1));
     }
 #undef GALV_H2D
     int32_t* d_C = (sh->flags & GALV_STORE_C_FULL) ? reinterpret_cast<int32_t*>(d + ar.C) : nullptr;

@@ -22,7 +22,7 @@ __device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v)
     return v;
 }
 
-__global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch,
+__global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, long long trans_inst, long long trans_layer,
                                  const int32_t* __restrict__ L, const int32_t* __restrict__ time_q,
                                  const int32_t* __restrict__ mem_q, const int32_t* __restrict__ trans_q,
                                  const int32_t* __restrict__ C, const uint8_t* __restrict__ A,
@@ -73,7 +73,7 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch,
 
     const int32_t* tq = time_q + (size_t)i * Lmax * S;
     const int32_t* mq = mem_q + (size_t)i * Lmax * S;
-    const int32_t* T = trans_q + (size_t)i * S * S;
+    const int32_t* T0 = trans_q + (size_t)i * trans_inst;
     int m = bud;
     long long used = 0;
     for (int l = Li - 1; l >= 0; --l) {
@@ -87,6 +87,7 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch,
         } else {
             const int target = C[((size_t)i * Lmax + l) * slice + (size_t)s * m_pitch + m] - tq[l * S + s];
             const int32_t* prev = C + ((size_t)i * Lmax + (l - 1)) * slice + (m - mm);
+            const int32_t* T = T0 + (size_t)l * trans_layer;       // paid between layers l-1 and l
             sp = 255;
             for (int base = 0; base < S; base += 32) {
                 const int k = base + lane;
@@ -119,7 +120,7 @@ cudaError_t galv_backtrack_launch(const galv_shape* sh, const int32_t* L, const 
 {
     const int warps = 4;
     backtrack_kernel<<<(sh->B + warps - 1) / warps, warps * 32, 0, st>>>(
-        sh->B, sh->Lmax, sh->S, sh->M, sh->m_pitch, L, time_q, mem_q, trans_q, C, A, C_last, budget,
+        sh->B, sh->Lmax, sh->S, sh->M, sh->m_pitch, galv_trans_inst(sh), galv_trans_layer(sh), L, time_q, mem_q, trans_q, C, A, C_last, budget,
         opt_cost, plan, mem_used, status);
     return cudaGetLastError();
 }

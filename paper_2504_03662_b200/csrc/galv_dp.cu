@@ -111,7 +111,9 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 // ---------------------------------------------------------------- validation / schedule
 
 // One CTA per instance: entries >= 0, L in range, worst-case path sum below kInf.
-__global__ void validate_kernel(int B, int Lmax, int S, int M, const int32_t* __restrict__ L,
+// tl: entries between the transition matrices of consecutive layers (0: one matrix per instance; S*S: matrix l
+// is paid between layers l-1 and l, matrix 0 unused).
+__global__ void validate_kernel(int B, int Lmax, int S, int M, long long tl, const int32_t* __restrict__ L,
                                 const int32_t* __restrict__ time_q, const int32_t* __restrict__ mem_q,
                                 const int32_t* __restrict__ trans_q, int32_t* __restrict__ status,
                                 int32_t* __restrict__ maxmem, int32_t* __restrict__ minmem_l, int32_t* __restrict__ front)
@@ -140,9 +142,10 @@ __global__ void validate_kernel(int B, int Lmax, int S, int M, const int32_t* __
         }
         sum += mx;
     }
-    const int32_t* x = trans_q + (size_t)i * S * S;
-    for (int k = threadIdx.x; k < S * S; k += blockDim.x) {
-        const int v = x[k];
+    const int32_t* x = trans_q + (size_t)i * (tl ? (size_t)Lmax * S * S : (size_t)S * S);
+    const int xl0 = tl ? 1 : 0, xl1 = tl ? Li : 1;            // matrices in use
+    for (int k = threadIdx.x; k < (xl1 - xl0) * S * S; k += blockDim.x) {
+        const int v = x[(size_t)xl0 * S * S + k];
         bad |= (v < 0);
         tmax = max(tmax, v);
     }
@@ -245,7 +248,7 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
     const size_t slice = (size_t)a.S * a.m_pitch;
     const int32_t* prev = a.C ? a.C + ((size_t)i * a.Lmax + (l - 1)) * slice : a.roll + ((size_t)((l - 1) & 1) * a.B + i) * slice;
     int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
-    const int32_t* T = a.trans_q + (size_t)i * a.S * a.S;
+    const int32_t* T = a.trans_q + (size_t)i * a.trans_inst + (size_t)l * a.trans_layer;
     const int mm = a.mem_q[((size_t)i * a.Lmax + l) * a.S + s];
     const int tt = a.time_q[((size_t)i * a.Lmax + l) * a.S + s];
     int best = kInf, arg = 255;
@@ -427,7 +430,8 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
             const int yc = row0 + i * inst_rows;
-            const int32_t* T = a.trans_q + (size_t)i * S * S + sb0;
+            const int32_t* T = a.trans_q + (size_t)i * a.trans_inst + (size_t)l * a.trans_layer + sb0;
+            const int yt = a.trans_layer ? (i * a.Lmax + l) * S : i * S;     // row of trans(0, .) in the tensor map
             // a tile wholly below the previous layer's feasibility frontier reads nothing but +inf: no loads
             const bool skip = a.front && m0 + TMB - 1 < a.front[(size_t)i * a.Lmax + (l - 1)];
             for (int kc = 0; kc < NKC; ++kc, ++n) {
@@ -460,7 +464,7 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
 #pragma unroll
                     for (int bx = 0; bx < NBOX; ++bx)
                         tma_load_2d(cs + bx * KS * BOXC, &map_c, m0 + bx * BOXC, yc + k0, &full_bar[st]);
-                    if (tma_t) tma_load_2d(ts, &map_t, sb0, i * S + k0, &full_bar[st]);
+                    if (tma_t) tma_load_2d(ts, &map_t, sb0, yt + k0, &full_bar[st]);
                 }
                 __syncwarp();
             }
@@ -937,7 +941,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     if (reference) { pl.tmb = 256; pl.ntiles_m = (a.M + 256) / 256; }
     e = cudaMemsetAsync(a.minmem_l, 0x7f, (size_t)(Lmax + 1) * 4, st);
     if (e != cudaSuccess) return e;
-    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1, a.minmem_l,
+    validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, (long long)a.trans_layer, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1, a.minmem_l,
                                        (sh->flags & GALV_SKIP_INFEASIBLE) ? a.front : nullptr);
     schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.M, pl.tmb, pl.ntiles_m, a.L, a.status, a.order, a.nactive, a.scratch,
                                          a.minmem_l, a.ntiles);
@@ -966,7 +970,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
         const size_t rows = a.C ? (size_t)B * Lmax * S : (size_t)2 * B * S;
         if ((e = encode_2d(&maps[0], a.C ? (void*)a.C : (void*)a.roll, (size_t)a.m_pitch, rows, boxc, pl.ks)) != cudaSuccess) return e;
         if (pl.tma_t &&
-            (e = encode_2d(&maps[1], (void*)a.trans_q, (size_t)S, (size_t)B * S, pl.sb, pl.ks)) != cudaSuccess) return e;
+            (e = encode_2d(&maps[1], (void*)a.trans_q, (size_t)S, (size_t)B * (a.trans_layer ? Lmax : 1) * S, pl.sb, pl.ks)) != cudaSuccess) return e;
     }
     // All layers in one cooperative launch when the grid's CTAs can be co-resident (they wait on one
     // another's tiles); with an argmin table, on request, or for the reference kernel: one launch per layer.

@@ -20,7 +20,7 @@ namespace {
 
 // One warp per instance: cost(p) = sum_l time(l,p_l) + sum_{l>=1} trans(p_{l-1},p_l), mem = sum_l mem(l,p_l).
 // -1 for both when the plan has an entry outside 0..S-1 within the instance's layers.
-__global__ void plan_cost_kernel(int B, int Lmax, int S, const int32_t* __restrict__ L, const int32_t* __restrict__ time_q,
+__global__ void plan_cost_kernel(int B, int Lmax, int S, long long trans_inst, long long trans_layer, const int32_t* __restrict__ L, const int32_t* __restrict__ time_q,
                                  const int32_t* __restrict__ mem_q, const int32_t* __restrict__ trans_q,
                                  const int32_t* __restrict__ plan, long long* __restrict__ cost, long long* __restrict__ mem_total)
 {
@@ -38,7 +38,7 @@ __global__ void plan_cost_kernel(int B, int Lmax, int S, const int32_t* __restri
             u += mem_q[((size_t)i * Lmax + l) * S + p];
             if (l >= 1) {
                 const int q = plan[(size_t)i * Lmax + l - 1];
-                if (q >= 0 && q < S) c += trans_q[((size_t)i * S + q) * S + p];
+                if (q >= 0 && q < S) c += trans_q[(size_t)i * trans_inst + (size_t)l * trans_layer + (size_t)q * S + p];
             }
         }
 #pragma unroll
@@ -63,7 +63,7 @@ int galv_plan_cost(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const 
     if (!ctx) return GALV_ERR_INVALID_ARG;
     if (!sh || sh->B < 1 || sh->S < 1 || sh->Lmax < 1 || !L || !time_q || !mem_q || !trans_q || !plan || !cost || !mem_total)
         return galv_set_error(ctx, GALV_ERR_INVALID_ARG, "galv_plan_cost: bad shape or NULL pointer");
-    plan_cost_kernel<<<(sh->B + 3) / 4, 128, 0, (cudaStream_t)stream>>>(sh->B, sh->Lmax, sh->S, L, time_q, mem_q, trans_q, plan,
+    plan_cost_kernel<<<(sh->B + 3) / 4, 128, 0, (cudaStream_t)stream>>>(sh->B, sh->Lmax, sh->S, galv_trans_inst(sh), galv_trans_layer(sh), L, time_q, mem_q, trans_q, plan,
                                                                        reinterpret_cast<long long*>(cost),
                                                                        reinterpret_cast<long long*>(mem_total));
     const cudaError_t e = cudaGetLastError();

@@ -41,6 +41,8 @@ struct DpArgs {
     const int32_t* time_q;
     const int32_t* mem_q;
     const int32_t* trans_q;
+    long long trans_inst;   // entries per instance in trans_q: S*S, or Lmax*S*S with one matrix per layer
+    long long trans_layer;  // entries between the matrices of consecutive layers: 0 or S*S
     int32_t* C;          // full table or NULL
     uint8_t* A;          // argmin table or NULL
     int32_t* C_last;
@@ -68,6 +70,8 @@ WsLayout galv_ws_layout(const galv_shape* sh);
 bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* plan);
 cudaError_t galv_dp_configure(const galv_ctx* ctx);
 cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a, cudaStream_t st);
+inline long long galv_trans_layer(const galv_shape* sh) { return (sh->flags & GALV_TRANS_PER_LAYER) ? (long long)sh->S * sh->S : 0; }
+inline long long galv_trans_inst(const galv_shape* sh) { return (long long)sh->S * sh->S * ((sh->flags & GALV_TRANS_PER_LAYER) ? sh->Lmax : 1); }
 cudaError_t galv_backtrack_launch(const galv_shape* sh, const int32_t* L, const int32_t* time_q,
                                   const int32_t* mem_q, const int32_t* trans_q, const int32_t* C,
                                   const uint8_t* A, const int32_t* C_last, const int32_t* budget,

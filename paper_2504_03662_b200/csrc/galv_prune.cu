@@ -102,6 +102,8 @@ int galv_prune_strategies(galv_ctx* ctx, const galv_shape* sh, const int32_t* L,
     if (!ctx) return GALV_ERR_INVALID_ARG;
     if (!sh || sh->B < 1 || sh->S < 1 || sh->S > 256 || sh->Lmax < 1 || !L || !time_q || !mem_q || !trans_q || !keep || !map || !S_kept)
         return galv_set_error(ctx, GALV_ERR_INVALID_ARG, "galv_prune_strategies: bad shape or NULL pointer");
+    if (sh->flags & GALV_TRANS_PER_LAYER)
+        return galv_set_error(ctx, GALV_ERR_INVALID_ARG, "galv_prune_strategies: one transition matrix per instance only (no GALV_TRANS_PER_LAYER)");
     cudaStream_t st = (cudaStream_t)stream;
     prune_kernel<<<sh->S, 256, 0, st>>>(sh->B, sh->Lmax, sh->S, L, time_q, mem_q, trans_q, keep);
     prune_map_kernel<<<1, 32, 0, st>>>(sh->S, keep, map, S_kept);
@@ -115,8 +117,8 @@ int galv_compact_tables(galv_ctx* ctx, const galv_shape* sh, int32_t S_kept, con
 {
     if (!ctx) return GALV_ERR_INVALID_ARG;
     if (!sh || sh->B < 1 || sh->S < 1 || sh->Lmax < 1 || S_kept < 1 || S_kept > sh->S || !map || !time_q || !mem_q || !trans_q ||
-        !time_out || !mem_out || !trans_out)
-        return galv_set_error(ctx, GALV_ERR_INVALID_ARG, "galv_compact_tables: bad shape, S_kept outside 1..S, or NULL pointer");
+        !time_out || !mem_out || !trans_out || (sh->flags & GALV_TRANS_PER_LAYER))
+        return galv_set_error(ctx, GALV_ERR_INVALID_ARG, "galv_compact_tables: bad shape, S_kept outside 1..S, per-layer trans, or NULL pointer");
     const long long n = (long long)sh->B * sh->Lmax * S_kept + (long long)sh->B * S_kept * S_kept;
     compact_kernel<<<blocks_for(n), 256, 0, (cudaStream_t)stream>>>(sh->B, sh->Lmax, sh->S, S_kept, map, time_q, mem_q, trans_q,
                                                                    time_out, mem_out, trans_out);

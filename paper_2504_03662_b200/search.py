@@ -26,6 +26,9 @@ class SearchBuffers:
         self.galv, self.w, self.flags = galv, w, flags
         dev = torch.device(device or f"cuda:{galv.device}")
         self.dev = dev
+        if w.trans_q is not None and w.trans_q.ndim == 4:          # one transition matrix per layer
+            flags |= gb.TRANS_PER_LAYER
+        self.flags = flags
         self.shape = gb.make_shape(w.B, w.Lmax, w.S, w.M, flags)
         B, Lm, S, P = w.B, w.Lmax, w.S, self.shape.m_pitch
         i32 = dict(dtype=torch.int32, device=dev)
@@ -99,6 +102,8 @@ class HostSearch:
 
     def __init__(self, galv: gb.Galv, w: Workload, flags: int = gb.STORE_C_FULL):
         self.galv, self.w = galv, w
+        if w.trans_q is not None and w.trans_q.ndim == 4:          # one transition matrix per layer
+            flags |= gb.TRANS_PER_LAYER
         self.shape = gb.make_shape(w.B, w.Lmax, w.S, w.M, flags)
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
         self.L = pin(np.ascontiguousarray(w.L, np.int32))
