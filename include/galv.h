@@ -270,6 +270,25 @@ int galv_graph_create(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
 int galv_graph_launch(galv_ctx* ctx, galv_graph* graph, void* stream);
 int galv_graph_destroy(galv_graph* graph);
 
+/*
+ * Stage partitioning (Sections 2-3: layers are spread over pipeline stages so that the stages are
+ * balanced, and re-cut when one becomes the bottleneck).  Build the batch with one instance per
+ * start layer a (its layers are a, a+1, ..., so B = Lmax = Lm and L[a] = Lm - a) and search it with
+ * the full table kept; galv_layer_optima then reads out, for every instance and layer,
+ *   opt_l[i][l] = min_s C[i][l][s][budget_i]      (GALV_INF beyond L[i] and for flagged instances),
+ * i.e. opt_l[a][n-1] = optimum of the stage made of layers a .. a+n-1.  budget NULL: M.
+ * galv_stage_partition cuts layers 0..Lm-1 into P consecutive stages minimising the slowest stage:
+ *   f[1][b] = opt(0,b),  f[k][b] = min_{k-1 <= a < b} max(f[k-1][a], opt(a,b)),  range_opt = opt_l.
+ * cuts int32 [P+1]: 0 = cuts[0] < ... < cuts[P] = Lm (walking back from the end, the lowest a that
+ * attains f[k][b]); bottleneck int32 [1] = f[P][Lm]; GALV_INF and cuts = -1 when nothing is
+ * feasible or P > Lm.  (P+1)*(Lm+1) must fit one CTA's shared memory (about 28 000 entries).
+ * All device pointers.
+ */
+int galv_layer_optima(galv_ctx* ctx, const galv_shape* shape, const int32_t* L, const int32_t* C,
+                      const int32_t* budget, const int32_t* status, int32_t* opt_l, void* stream);
+int galv_stage_partition(galv_ctx* ctx, int32_t Lm, int32_t P, const int32_t* range_opt,
+                         int32_t* cuts, int32_t* bottleneck, void* stream);
+
 /* Bytes of device arena galv_search_host needs (0 on invalid shape). */
 size_t galv_search_host_arena_bytes(const galv_ctx* ctx, const galv_shape* shape, int with_model);
 

@@ -346,3 +346,49 @@ void orc_prune(int B, int Lmax, int S, const int32_t *L, const int32_t *time, co
         }
     }
 }
+
+/* ------------------------------------------------------------------ stage partitioning
+ *
+ * The model's layers are cut into P consecutive pipeline stages (Section 2 and Section 3 of the
+ * paper: layers are distributed over stages so that the work per stage is balanced, and re-cut when
+ * a stage becomes the bottleneck).  range_opt[a][n-1] is the optimum of the layer-wise search for the
+ * stage made of layers a .. a+n-1 (ORC_INF when nothing fits); a pipeline runs at the pace of its
+ * slowest stage, so the cut minimises the largest stage optimum:
+ *   f[1][b] = opt(0,b),   f[k][b] = min_{k-1 <= a < b} max( f[k-1][a], opt(a,b) ).
+ * cuts[0] = 0 < cuts[1] < ... < cuts[P] = Lm.  Several cuts can share the optimal bottleneck; the
+ * one reported is the one the recurrence defines: walking back from the end, the lowest a attaining
+ * f[k][b] is taken, so every prefix of the partition is itself cut optimally (not merely below the
+ * bottleneck).  bottleneck = ORC_INF and cuts = -1 when no partition is feasible or P > Lm.
+ */
+void orc_stage_partition(int Lm, int P, const int32_t *range_opt, int32_t *cuts, int32_t *bottleneck)
+{
+    for (int k = 0; k <= P; k++) cuts[k] = -1;
+    *bottleneck = ORC_INF;
+    if (P < 1 || P > Lm) return;
+    int32_t *f = (int32_t *)malloc((size_t)(P + 1) * (Lm + 1) * sizeof(int32_t));
+    int32_t *g = (int32_t *)malloc((size_t)(P + 1) * (Lm + 1) * sizeof(int32_t));
+    for (int k = 1; k <= P; k++)
+        for (int b = 0; b <= Lm; b++) {
+            int32_t best = ORC_INF, arg = -1;
+            if (b >= k) {
+                if (k == 1) { best = range_opt[0 * Lm + (b - 1)]; arg = 0; }
+                else
+                    for (int a = k - 1; a < b; a++) {
+                        int32_t left = f[(k - 1) * (Lm + 1) + a], here = range_opt[a * Lm + (b - a - 1)];
+                        int32_t v = left > here ? left : here;
+                        if (v < best) { best = v; arg = a; }
+                    }
+            }
+            if (best >= ORC_INF) { best = ORC_INF; arg = -1; }
+            f[k * (Lm + 1) + b] = best;
+            g[k * (Lm + 1) + b] = arg;
+        }
+    *bottleneck = f[P * (Lm + 1) + Lm];
+    if (*bottleneck < ORC_INF) {
+        int b = Lm;
+        for (int k = P; k >= 1; k--) { cuts[k] = b; b = g[k * (Lm + 1) + b]; }
+        cuts[0] = 0;
+    }
+    free(f);
+    free(g);
+}

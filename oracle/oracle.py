@@ -151,3 +151,13 @@ def prune(L, time, mem, trans):
     keep = np.empty(S, np.int32)
     lib().orc_prune(B, Lmax, S, pl, pt, pm, px, keep.ctypes.data_as(C.c_void_p))
     return keep
+
+
+def stage_partition(range_opt, P: int):
+    """(bottleneck, cuts[P+1]) for range_opt [Lm][Lm] (row a, column n-1: optimum of layers a..a+n-1)."""
+    ro, pr = _i32(range_opt)
+    Lm = ro.shape[0]
+    assert ro.shape == (Lm, Lm)
+    cuts = np.empty(P + 1, np.int32); bn = C.c_int32()
+    lib().orc_stage_partition(Lm, P, pr, cuts.ctypes.data_as(C.c_void_p), C.byref(bn))
+    return bn.value, cuts

@@ -27,7 +27,7 @@ EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "g
            "galv_dp_workspace_bytes", "galv_dp_search", "galv_backtrack", "galv_search_host_arena_bytes",
            "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_dp_search_static", "galv_select_best", "galv_prune_strategies",
            "galv_compact_tables", "galv_expand_plan", "galv_plan_cost", "galv_graph_create", "galv_graph_launch",
-           "galv_graph_destroy")
+           "galv_graph_destroy", "galv_layer_optima", "galv_stage_partition")
 
 
 class galv_shape(C.Structure):
@@ -74,6 +74,8 @@ def load_library() -> C.CDLL:
     lib.galv_graph_create.argtypes = [vp, shp, vp, vp, i64, vp, vp] + [vp] * 7 + [sz] + [vp] * 6 + [C.POINTER(vp)]
     lib.galv_graph_launch.argtypes = [vp, vp, vp]
     lib.galv_graph_destroy.argtypes = [vp]
+    lib.galv_layer_optima.argtypes = [vp, shp] + [vp] * 6
+    lib.galv_stage_partition.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, vp, vp]
     lib.galv_search_host_arena_bytes.argtypes = [vp, shp, C.c_int]
     lib.galv_search_host_arena_bytes.restype = sz
     lib.galv_search_host.argtypes = [vp, shp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -181,6 +183,13 @@ class Galv:
 
     def galv_graph_destroy(self, graph):
         self.lib.galv_graph_destroy(graph)
+
+    def galv_layer_optima(self, shape, L, Ct, budget, status, opt_l):
+        self._check(self.lib.galv_layer_optima(self.h, C.byref(shape), _ptr(L), _ptr(Ct), _ptr(budget), _ptr(status),
+                                               _ptr(opt_l), _stream()))
+
+    def galv_stage_partition(self, Lm, P, range_opt, cuts, bottleneck):
+        self._check(self.lib.galv_stage_partition(self.h, Lm, P, _ptr(range_opt), _ptr(cuts), _ptr(bottleneck), _stream()))
 
     def galv_backtrack(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, budget, opt_cost, plan, mem_used, status):
         self._check(self.lib.galv_backtrack(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),

@@ -1,0 +1,152 @@
+"""Stage partitioning: oracle pins (CPU) and GPU parity, including the suffix-batch construction."""
+import itertools
+
+import numpy as np
+import pytest
+
+from paper_2504_03662_b200 import inputs
+
+INF = 2 ** 30 - 1
+
+
+def random_range_opt(seed, Lm, additive=False, holes=0.0):
+    rng = np.random.default_rng(seed)
+    ro = np.full((Lm, Lm), INF, np.int32)
+    layer = rng.integers(1, 100, size=Lm)
+    for a in range(Lm):
+        for n in range(1, Lm - a + 1):
+            v = int(layer[a:a + n].sum()) if additive else int(layer[a:a + n].sum() + rng.integers(0, 30))
+            ro[a, n - 1] = INF if rng.random() < holes else v
+    return ro
+
+
+def brute_bottleneck(ro, P):
+    Lm = ro.shape[0]
+    best = INF
+    for inner in itertools.combinations(range(1, Lm), P - 1):
+        c = (0,) + inner + (Lm,)
+        best = min(best, max(int(ro[c[k], c[k + 1] - c[k] - 1]) for k in range(P)))
+    return best
+
+
+def check_cuts(ro, P, bn, cuts):
+    Lm = ro.shape[0]
+    if bn >= INF:
+        assert (cuts == -1).all()
+        return
+    assert cuts[0] == 0 and cuts[P] == Lm and (np.diff(cuts) >= 1).all()
+    assert max(int(ro[cuts[k], cuts[k + 1] - cuts[k] - 1]) for k in range(P)) == bn
+
+
+def test_uniform_layers_closed_form(orc):
+    # every layer costs 5 and stage cost is additive: the best bottleneck is 5 * ceil(Lm / P)
+    for Lm, P in ((7, 3), (12, 4), (10, 1), (9, 9), (5, 2)):
+        ro = np.full((Lm, Lm), INF, np.int32)
+        for a in range(Lm):
+            for n in range(1, Lm - a + 1):
+                ro[a, n - 1] = 5 * n
+        bn, cuts = orc.stage_partition(ro, P)
+        assert bn == 5 * -(-Lm // P)
+        check_cuts(ro, P, bn, cuts)
+    assert orc.stage_partition(ro, 6)[0] == INF              # more stages than layers
+
+
+def test_hand_example(orc):
+    # four layers with stage optima opt(a,n): a heavy layer 2 should sit alone.
+    # layers cost 2, 3, 10, 1 (additive): P=3 -> [0,2,3,4]: stages 5 | 10 | 1 -> bottleneck 10
+    cost = [2, 3, 10, 1]
+    ro = np.full((4, 4), INF, np.int32)
+    for a in range(4):
+        for n in range(1, 5 - a):
+            ro[a, n - 1] = sum(cost[a:a + n])
+    bn, cuts = orc.stage_partition(ro, 3)
+    # f[2][2] = min(max(2,3)) = 3 at a=1; f[2][3] = min(max(2,13), max(5,10)) = 10 at a=2;
+    # f[3][4] = min over a in {2,3}: max(f[2][2]=3, opt(2,4)=11) = 11, max(f[2][3]=10, opt(3,4)=1) = 10 -> a=3
+    assert bn == 10 and cuts.tolist() == [0, 2, 3, 4]
+    assert orc.stage_partition(ro, 2)[0] == 11               # 5 | 11
+    bn4, cuts4 = orc.stage_partition(ro, 4)
+    assert bn4 == 10 and cuts4.tolist() == [0, 1, 2, 3, 4]
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_oracle_against_all_cuts(orc, seed):
+    rng = np.random.default_rng(seed)
+    Lm = int(rng.integers(1, 10)); P = int(rng.integers(1, min(Lm, 5) + 1))
+    ro = random_range_opt(seed, Lm, additive=seed % 2 == 0, holes=0.15 if seed % 3 == 0 else 0.0)
+    bn, cuts = orc.stage_partition(ro, P)
+    assert bn == brute_bottleneck(ro, P)
+    check_cuts(ro, P, bn, cuts)
+    if bn < INF and P > 1:
+        # every prefix of the reported partition is itself cut optimally
+        for k in range(1, P):
+            sub = ro[:cuts[k], :cuts[k]]
+            assert orc.stage_partition(sub, k)[0] == max(int(ro[cuts[j], cuts[j + 1] - cuts[j] - 1]) for j in range(k))
+
+
+def suffix_batch(base: inputs.Workload) -> inputs.Workload:
+    """One instance per start layer a of the single-instance workload `base`: layers a, a+1, ..."""
+    Lm, S = base.Lmax, base.S
+    t = np.zeros((Lm, Lm, S), np.int32); m = np.zeros_like(t)
+    for a in range(Lm):
+        t[a, :Lm - a] = base.time_q[0, a:]
+        m[a, :Lm - a] = base.mem_q[0, a:]
+    x = np.repeat(base.trans_q[:1], Lm, 0)
+    return inputs.Workload(base.name + "_suffixes", Lm, Lm, S, base.M, (Lm - np.arange(Lm)).astype(np.int32), t, m, x)
+
+
+@pytest.mark.gpu
+def test_gpu_partition_matches_oracle(orc):
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    galv = gb.Galv(0)
+    try:
+        for seed, (Lm, P) in enumerate([(1, 1), (9, 3), (40, 8), (160, 16), (7, 9)]):
+            ro = random_range_opt(100 + seed, Lm, holes=0.05 if seed == 2 else 0.0)
+            d = torch.from_numpy(ro).cuda()
+            cuts = torch.empty(P + 1, dtype=torch.int32, device="cuda"); bn = torch.empty(1, dtype=torch.int32, device="cuda")
+            galv.galv_stage_partition(Lm, P, d, cuts, bn)
+            torch.cuda.synchronize()
+            rb, rc = orc.stage_partition(ro, P)
+            assert bn.item() == rb and (cuts.cpu().numpy() == rc).all()
+    finally:
+        galv.close()
+
+
+@pytest.mark.gpu
+def test_gpu_search_optima_partition_end_to_end(orc):
+    """Heterogeneous 14-layer stack: suffix batch -> search -> per-range optima -> 4 balanced stages."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    galv = gb.Galv(0)
+    try:
+        base = inputs.random_tables(9, 1, 14, 10, 160, mem_lo=2, mem_hi=30, time_hi=5000, trans_hi=300)
+        base.time_q[0, ::3] *= 4                                  # every third layer is heavy
+        w = suffix_batch(base)
+        sb = SearchBuffers(galv, w, gb.STORE_C_FULL)
+        sb.dp_search()
+        opt_l = torch.empty(w.B, w.Lmax, dtype=torch.int32, device=sb.dev)
+        galv.galv_layer_optima(sb.shape, sb.L, sb.C, None, sb.status, opt_l)
+        P = 4
+        cuts = torch.empty(P + 1, dtype=torch.int32, device=sb.dev); bn = torch.empty(1, dtype=torch.int32, device=sb.dev)
+        galv.galv_stage_partition(w.Lmax, P, opt_l, cuts, bn)
+        torch.cuda.synchronize()
+        # oracle: the same optima from its own tables, then its own partition
+        ro = np.full((w.Lmax, w.Lmax), INF, np.int32)
+        for a in range(w.Lmax):
+            n = w.Lmax - a
+            Ct, _ = orc.dp(w.time_q[a, :n], w.mem_q[a, :n], w.trans_q[a], w.M, want_A=False)
+            ro[a, :n] = Ct[:, w.M, :].min(axis=1)
+        assert (opt_l.cpu().numpy() == ro).all()
+        rb, rc = orc.stage_partition(ro, P)
+        assert bn.item() == rb and (cuts.cpu().numpy() == rc).all() and rb < INF
+        # a tighter budget query through the same tables
+        bud = torch.full((w.B,), 60, dtype=torch.int32, device=sb.dev)
+        galv.galv_layer_optima(sb.shape, sb.L, sb.C, bud, sb.status, opt_l)
+        torch.cuda.synchronize()
+        for a in (0, 5):
+            n = w.Lmax - a
+            Ct, _ = orc.dp(w.time_q[a, :n], w.mem_q[a, :n], w.trans_q[a], w.M, want_A=False)
+            assert (opt_l[a, :n].cpu().numpy() == Ct[:, 60, :].min(axis=1)).all()
+    finally:
+        galv.close()
