@@ -190,9 +190,11 @@ __global__ void validate_kernel(int B, int Lmax, int S, int M, long long tl, con
 // ntiles[l] = tiles of tmb columns per instance that can store anything in layer l: column m' lands at
 // m' + mem(l,s) <= M, so tiles starting above M - (smallest mem of the layer) are left out (at least one
 // tile stays: it also writes the cells no column maps to).
-__global__ void schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, const int32_t* __restrict__ L,
+// istart[l] = work items (instance, tile, s-block) of layers 1 .. l-1: the items of all layers in one sequence.
+__global__ void schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, int nsb, const int32_t* __restrict__ L,
                                 const int32_t* __restrict__ status, int32_t* __restrict__ order, int32_t* __restrict__ nactive,
-                                int32_t* __restrict__ scratch, const int32_t* __restrict__ minmem_l, int32_t* __restrict__ ntiles)
+                                int32_t* __restrict__ scratch, const int32_t* __restrict__ minmem_l, int32_t* __restrict__ ntiles,
+                                long long* __restrict__ istart, int32_t* __restrict__ tcount)
 {
     int32_t* hist = scratch;
     int32_t* fill = scratch + Lmax + 2;
@@ -213,6 +215,24 @@ __global__ void schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, c
         int nt = 1;
         if (l < Lmax && minmem_l[l] <= M) nt = min(ntiles_m, (M - minmem_l[l]) / tmb + 1);
         ntiles[l] = max(1, nt);
+    }
+    __syncthreads();
+    // tcount[l][t] = layers 1..l whose items include tile t
+    for (int t = threadIdx.x; t < ntiles_m; t += blockDim.x) {
+        int run = 0;
+        tcount[t] = 0;
+        for (int l = 1; l < Lmax; ++l) {
+            run += t < ntiles[l];
+            tcount[(size_t)l * ntiles_m + t] = run;
+        }
+    }
+    if (threadIdx.x == 0) {
+        long long run = 0;
+        istart[0] = 0;
+        for (int l = 1; l <= Lmax; ++l) {
+            istart[l] = run;
+            if (l < Lmax) run += (long long)nactive[l] * ntiles[l] * nsb;
+        }
     }
 }
 
@@ -269,10 +289,12 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 
 // ---------------------------------------------------------------- tiled layer kernel
 //
-// Work items are (instance, m'-tile, s-block); every CTA owns a contiguous run of them, so
-// consecutive items mostly share the instance (its trans rows stay in L2).  Warp roles:
-//   warp NC (producer): for every chunk (item, k-chunk of s') waits for a free stage, then
-//       bulk-copies KS rows of the previous layer's slice and the matching rows of trans into it;
+// Work items are (layer, instance, m'-tile, s-block), numbered layer by layer.  CTAs take them one
+// at a time from a global counter, so the SMs stay evenly loaded whatever the items weigh, and items
+// taken at about the same time mostly share the instance (its trans rows stay in L2).  Warp roles:
+//   warp NC (producer): takes the next item and posts its record in a small ring in shared memory
+//       for the other roles; then for every chunk (item, k-chunk of s') waits for a free stage and
+//       copies KS rows of the previous layer's slice and the matching rows of trans into it (TMA);
 //   warp NC+1 (helper): stages each item's record (mem and time row of the s-block, instance)
 //       next to the item's last chunk, and writes the cells no column maps to (m < mem(l,s))
 //       and the pad columns;
@@ -304,26 +326,14 @@ __device__ __forceinline__ ItemPos item_at(long long item, int nt, int nsb) {
     p.sb = r - p.mt * nsb;
     return p;
 }
-__device__ __forceinline__ void item_next(ItemPos& p, int nt, int nsb) {
-    if (++p.sb == nsb) { p.sb = 0; if (++p.mt == nt) { p.mt = 0; ++p.oi; } }
-}
+
+// Item records in flight: the producer runs at most (stages + 3) items ahead of the store warp.
+constexpr int kDescRing = 16;
 
 // Shared memory: NST stages of [KS][TMB] previous-layer values + [KS][SB] trans values, then per
 // stage a small record the producer fills for the item whose last chunk sits in that stage:
 // mem(l,s) and time(l,s) of the s-block and the instance index; then the staging tile of the
 // outputs and its header.
-// Items are dealt to CTAs by weight, not by count: a full tile weighs 64, the ragged last tile of
-// an instance (fewer than TMB columns) in proportion to its 32-column groups.  Returns the first
-// item whose cumulative weight reaches `target`.
-__device__ __forceinline__ long long item_at_weight(long long target, int nt, int nsb, int wr) {
-    const long long full = (long long)(nt - 1) * nsb * 64;                 // weight of an instance's full tiles
-    const long long per = full + (long long)nsb * wr;
-    const long long oi = target / per;
-    const long long rem = target - oi * per;
-    const long long idx = rem < full ? (rem + 63) / 64 : (nt - 1) * nsb + (rem - full + wr - 1) / wr;
-    return oi * nt * nsb + idx;
-}
-
 template <int TM, int NSG, int NMS, bool ARG, bool MULTI>
 __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
@@ -343,6 +353,8 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
     __shared__ __align__(8) uint64_t out_full, out_empty;  // staging tile written / drained
     __shared__ int fill_count;                             // helper -> store warp: first tiles whose unreachable cells are written
+    __shared__ int4 desc[kDescRing];                       // item records: layer (-1: no more items), instance, tile, s-block
+    __shared__ int desc_count;                             // records posted so far
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
@@ -353,18 +365,8 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
     // Layers l_first .. l_last-1.  One layer per launch, or all of them in one cooperative launch
     // (a.tile_done set): then an item of layer l starts once the tiles of layer l-1 it reads are
     // complete, which their store warps publish in a.tile_done (see the producer and the store warp).
-    // Every role walks the same sequence of (layer, item); this CTA's items of layer l:
-    auto layer_range = [&](int l, ItemPos& first, int& nt) -> int {  // first item, tiles per instance; returns how many items
-        nt = a.ntiles[l];
-        // weight of the last tile of an instance: its 32-column groups out of TMB/32, in 64ths
-        const int last_cols = min(TMB, M + 1 - (nt - 1) * TMB);
-        const int wr = max(1, ((last_cols + 31) / 32) * 64 / (TMB / 32));
-        const long long wtot = (long long)a.nactive[l] * pl.nsb * ((long long)(nt - 1) * 64 + wr);
-        const long long it0 = item_at_weight(wtot * blockIdx.x / gridDim.x, nt, pl.nsb, wr);
-        const long long it1 = item_at_weight(wtot * (blockIdx.x + 1) / gridDim.x, nt, pl.nsb, wr);
-        first = item_at(it0, nt, pl.nsb);
-        return (int)(it1 - it0);
-    };
+    // Items are handed out in increasing order and read only items of the layer before, so the
+    // lowest unfinished item can always run: the waits end.
 
     // stage: NBOX boxes of [KS][BOXC] previous-layer values, then [KS][SB] trans values; 128-byte multiples
     int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
@@ -379,6 +381,7 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         mbar_init(&out_full, NC);
         mbar_init(&out_empty, 1);
         fill_count = 0;
+        desc_count = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -393,17 +396,45 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         // up to the largest mem, the kdep before it
         const int kdep = tile_done ? (min(*a.maxmem, M) + TMB - 1) / TMB : 0;
         int n = 0;                                        // chunk counter
-        for (int l = l_first; l < l_last; ++l) {
-        ItemPos pos;
-        int nt;
-        const int nit = layer_range(l, pos, nt);
-        const int row0 = a.C ? (l - 1) * S : ((l - 1) & 1) * a.B * S;      // row of (instance 0, layer l-1, s'=0)
-        for (int q = 0; q < nit; ++q, item_next(pos, nt, pl.nsb)) {
-            const int i = a.order[pos.oi];
+        // this launch's items are g_base .. g_end-1 of the sequence over all layers
+        const long long g_base = a.istart[l_first], g_end = a.istart[l_last];
+        unsigned long long* const work = a.work + (MULTI ? 0 : l_first);
+        int l = l_first, nt = a.ntiles[l_first];          // layer of the item at hand (items arrive in increasing order)
+        long long lbeg = g_base, lend = a.istart[l_first + 1];
+        for (int it = 0;; ++it) {
+            long long g = 0;
+            if (lane == 0) g = g_base + (long long)atomicAdd(work, 1ull);
+            g = __shfl_sync(0xffffffffu, g, 0);
+            const bool last = g >= g_end;
+            ItemPos pos = {0, 0, 0};
+            int i = 0;
+            if (!last) {
+                while (g >= lend) { ++l; lbeg = lend; lend = a.istart[l + 1]; nt = a.ntiles[l]; }
+                pos = item_at(g - lbeg, nt, pl.nsb);
+                i = a.order[pos.oi];
+            }
+            if (lane == 0) {
+                desc[it % kDescRing] = make_int4(last ? -1 : l, i, pos.mt, pos.sb);
+                __threadfence_block();
+                *reinterpret_cast<volatile int*>(&desc_count) = it + 1;
+            }
+            __syncwarp();
+            if (last) {
+                // the consumers learn it through a stage that carries no data
+                const int st = n % NST;
+                if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+                if (lane == 0) mbar_arrive(&full_bar[st]);
+                return;
+            }
+            const int row0 = a.C ? (l - 1) * S : ((l - 1) & 1) * a.B * S;      // row of (instance 0, layer l-1, s'=0)
             const int m0 = pos.mt * TMB;
             if (MULTI && tile_done && l > 1) {
                 // bounded wait for the tiles of layer l-1 (all their s-blocks) this item reads
-                const int need = (l - 1) * pl.nsb;
+                // = s-blocks x the layers up to l-1 that ran the tile (trailing tiles are left out layer by layer)
+                const int32_t* const ran = a.tcount + (size_t)(l - 1) * pl.ntiles_m;
                 // one lane per tile polls (relaxed), then one acquire fence for the warp
                 bool ok = true;
                 const int tlast = min(pos.mt, a.ntiles[l - 1] - 1);      // tiles the previous layer did not run store nothing
@@ -412,6 +443,7 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                     if (t <= tlast) {
                         const int32_t* c = tile_done + (size_t)i * pl.ntiles_m + t;
                         WaitClock wc;
+                        const int need = ran[t] * pl.nsb;
                         while (ld_relaxed_gpu(c) < need) {
                             if (wc.expired()) { ok = false; break; }
                             __nanosleep(64);
@@ -469,18 +501,34 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 __syncwarp();
             }
         }
-        }
-        return;
     }
     if (warp == NC + 1) {
         // ------------------------------------------------------------ helper
         int n = 0;
-        for (int l = l_first; l < l_last; ++l) {
-        ItemPos pos;
-        int nt;
-        const int nit = layer_range(l, pos, nt);
-        for (int q = 0; q < nit; ++q, item_next(pos, nt, pl.nsb)) {
-            const int i = a.order[pos.oi];
+        for (int it = 0;; ++it) {
+            {
+                WaitClock wc;                             // the producer posts the item's record
+                while (*reinterpret_cast<volatile int*>(&desc_count) <= it) {
+                    if (wc.expired()) {
+                        if (lane == 0) atomicExch(a.err, 1);
+                        return;
+                    }
+                    __nanosleep(32);
+                }
+                __threadfence_block();
+            }
+            const int4 d = desc[it % kDescRing];
+            const int l = d.x, i = d.y;
+            ItemPos pos = {0, d.z, d.w};
+            if (l < 0) {
+                const int st = n % NST;
+                if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+                if (lane == 0) mbar_arrive(&full_bar[st]);
+                return;
+            }
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);
             const size_t qrow = ((size_t)i * a.Lmax + l) * S + sb0;
@@ -528,8 +576,6 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 }
             }
         }
-        }
-        return;
     }
 
     if (warp == NC + 2) {
@@ -550,16 +596,15 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 red_release_gpu_add(counter, 1);
             }
         };
-        for (int l = l_first; l < l_last; ++l) {
-        ItemPos pos;
-        int nt;
-        const int nit = layer_range(l, pos, nt);
-        for (int q = 0; q < nit; ++q, item_next(pos, nt, pl.nsb), ++it) {
+        for (;; ++it) {
             if (!mbar_wait(&out_full, it & 1)) {
                 if (lane == 0) atomicExch(a.err, 1);
                 return;
             }
-            const int i = hdr0[SB];
+            const int4 d = desc[it % kDescRing];
+            const int l = d.x, i = d.y;
+            if (l < 0) break;                                     // no more items
+            ItemPos pos = {0, d.z, d.w};
             const int m0 = pos.mt * TMB;
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);
@@ -584,9 +629,7 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
             if (lane == 0) mbar_arrive(&out_empty);
             if (MULTI && tile_done) {
                 // The previous item's bulk stores were issued a whole item ago: waiting for all groups
-                // but the newest costs nothing, and then that item is published.  The last item of a
-                // layer is published at once: other CTAs' first items of the next layer may need it,
-                // and this CTA's own next item may in turn wait for theirs.
+                // but the newest costs nothing, and then that item is published.
                 int32_t* mine = tile_done + (size_t)i * pl.ntiles_m + pos.mt;
                 if (pos.mt == 0) {                                // the helper's fill of this tile (it runs ahead)
                     ++nfill;
@@ -600,12 +643,19 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                     }
                 }
                 if (unpublished) { bulk_wait_all_but_last(); publish(unpublished); }
-                if (q + 1 == nit) { bulk_wait_all(); publish(mine); unpublished = nullptr; }
-                else unpublished = mine;
+                // Deferred only when this CTA's next item is known and sits in the same layer, so that
+                // it cannot itself be waiting for this tile; near a layer's end the tile is published at once.
+                bool defer = false;
+                if (*reinterpret_cast<volatile int*>(&desc_count) > it + 1) {
+                    __threadfence_block();
+                    defer = desc[(it + 1) % kDescRing].x == l;
+                }
+                if (defer) unpublished = mine;
+                else { bulk_wait_all(); publish(mine); unpublished = nullptr; }
             }
         }
-        }
         bulk_wait_all();
+        if (unpublished) publish(unpublished);
         return;
     }
 
@@ -614,15 +664,10 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
     int acc[TM][TS];
     int arg[ARG ? TM : 1][ARG ? TS : 1];
     (void)arg;
-    int n = 0, it = 0;
-    for (int l = l_first; l < l_last; ++l) {
-    ItemPos pos;
-    int nt;
-    const int nit = layer_range(l, pos, nt);
-    for (int q = 0; q < nit; ++q, item_next(pos, nt, pl.nsb), ++it) {
-        const int mw = pos.mt * TMB + ms * (32 * TM);       // first column of this warp
-        // 32-column groups of this warp that hold at least one column <= M
-        const int nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
+    int n = 0;
+    for (int it = 0;; ++it) {
+        int l = 0, mw = 0, nj = 0;
+        ItemPos pos = {0, 0, 0};
 #pragma unroll
         for (int j = 0; j < TM; ++j)
 #pragma unroll
@@ -636,6 +681,27 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
             if (!mbar_wait(&full_bar[st], (n / NST) & 1)) {
                 if (lane == 0) atomicExch(a.err, 1);
                 return;
+            }
+            if (kc == 0) {
+                // the item's record was posted before its first stage was filled
+                const int4 d = desc[it % kDescRing];
+                l = d.x;
+                if (l < 0) {
+                    // no more items: wake the store warp and leave.  Not before it has taken the previous
+                    // item: two completions of out_full in a row would hide the first from its parity wait.
+                    if (it > 0 && !mbar_wait(&out_empty, (it - 1) & 1)) {
+                        if (lane == 0) atomicExch(a.err, 1);
+                        return;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&out_full);
+                    return;
+                }
+                pos.mt = d.z;
+                pos.sb = d.w;
+                mw = pos.mt * TMB + ms * (32 * TM);         // first column of this warp
+                // 32-column groups of this warp that hold at least one column <= M
+                nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
             }
             const int k0 = kc * KS;
             // nothing but +inf to read (see the producer): the accumulators stay at +inf
@@ -759,7 +825,6 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         __syncwarp();
         if (lane == 0) mbar_arrive(&out_full);
     }
-    }
 }
 
 // C_last[i] = layer L[i]-1 of instance i (from the full table, or from the rolling buffer that
@@ -838,10 +903,12 @@ WsLayout galv_ws_layout(const galv_shape* sh)
     size_t off = 0;
     w.order = off;   off = align256(off + (size_t)sh->B * 4);
     w.nactive = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
-    w.scratch = off; off = align256(off + (size_t)2 * (sh->Lmax + 2) * 4);
+    w.scratch = off; off = align256(off + (size_t)4 * (sh->Lmax + 2) * 4);    // two int32 arrays, one 64-bit array
     w.err = off;     off = align256(off + 8);                  // error flag, largest mem
     w.minmem_l = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.ntiles = off;   off = align256(off + (size_t)(sh->Lmax + 1) * 4);
+    w.istart = off;   off = align256(off + (size_t)(sh->Lmax + 1) * 8);
+    w.tcount = off;   off = align256(off + (size_t)sh->Lmax * ((sh->M + 128) / 128) * 4);
     w.front = off;    off = align256(off + (size_t)sh->B * sh->Lmax * 4);
     w.tile_done = off; off = align256(off + (size_t)sh->B * ((sh->M + 128) / 128) * 4);   // per (instance, tile of >= 128 columns)
     w.roll = off;
@@ -930,7 +997,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
 {
     cudaError_t e;
     const int B = a.B, Lmax = a.Lmax, S = a.S;
-    e = cudaMemsetAsync(a.scratch, 0, (size_t)2 * (Lmax + 2) * 4, st);
+    e = cudaMemsetAsync(a.scratch, 0, (size_t)4 * (Lmax + 2) * 4, st);      // histogram, fill and work counters
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(a.err, 0, 8, st);
     if (e != cudaSuccess) return e;
@@ -943,8 +1010,8 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     if (e != cudaSuccess) return e;
     validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, (long long)a.trans_layer, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1, a.minmem_l,
                                        (sh->flags & GALV_SKIP_INFEASIBLE) ? a.front : nullptr);
-    schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.M, pl.tmb, pl.ntiles_m, a.L, a.status, a.order, a.nactive, a.scratch,
-                                         a.minmem_l, a.ntiles);
+    schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.M, pl.tmb, pl.ntiles_m, pl.nsb, a.L, a.status, a.order, a.nactive, a.scratch,
+                                         a.minmem_l, a.ntiles, a.istart, a.tcount);
     {
         int gx = (a.m_pitch + 255) / 256;
         if (gx > 8) gx = 8;

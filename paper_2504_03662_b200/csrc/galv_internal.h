@@ -49,13 +49,16 @@ struct DpArgs {
     int32_t* roll;       // [2][B][S][m_pitch] when C == NULL
     int32_t* order;      // [B]   valid instances, longest first
     int32_t* nactive;    // [Lmax+1] instances with L > l
-    int32_t* scratch;    // [2*(Lmax+2)] histogram / fill counters
+    int32_t* scratch;    // [2*(Lmax+2)] histogram / fill counters, then the work counters below (zeroed together)
+    unsigned long long* work;  // [Lmax+2] next item to hand out: [0] when all layers are one launch, else [l]
+    long long* istart;   // [Lmax+1] items of the layers before l (layer 1 starts at 0); [Lmax] = all items
     int32_t* err;        // device error flag
     int32_t* tile_done;  // [B][ntiles_m] finished items per (instance, tile); NULL when layers are separate launches
     int32_t* maxmem;     // largest mem over the valid instances (min(.., M+1))
     int32_t* minmem_l;   // [Lmax+1] smallest mem of each layer over the valid instances
     int32_t* front;      // [B][Lmax] feasibility frontier (sum of the layers' smallest mem), or NULL when tiles are never skipped
     int32_t* ntiles;     // [Lmax+1] tiles per instance that can store anything in layer l
+    int32_t* tcount;     // [Lmax][ntiles_m] layers 1..l whose items include tile t
     int32_t* status;
     int withhold;        // test hook: CTA 0 never loads its first chunk, so that the bounded waits run out
 };
@@ -64,7 +67,7 @@ struct DpArgs {
 int galv_set_error(galv_ctx* ctx, int code, const char* text);
 
 // workspace carve-up (offsets in bytes, all 256-aligned)
-struct WsLayout { size_t order, nactive, scratch, err, minmem_l, ntiles, front, tile_done, roll, total; };
+struct WsLayout { size_t order, nactive, scratch, err, minmem_l, ntiles, istart, tcount, front, tile_done, roll, total; };
 WsLayout galv_ws_layout(const galv_shape* sh);
 
 bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* plan);
