@@ -24,6 +24,7 @@
 #include <cuda.h>
 
 #include <cstring>
+#include <cstdlib>
 
 #include "galv_internal.h"
 
@@ -73,14 +74,21 @@ __device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t by
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all_but_last() { asm volatile("cp.async.bulk.wait_group 1;" ::: "memory"); }
-__device__ __forceinline__ int ld_relaxed_gpu(const int32_t* p) {
+__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
     int v;
-    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void red_release_gpu_add(int32_t* p, int v) {
-    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void red_relaxed_gpu_add(int32_t* p, int v) {
+    asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_release_cta(int* p, int v) {
+    asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_cta(const int* p) {
+    int v;
+    asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -303,6 +311,9 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 //       next item.  The SM's store port takes 32 bytes per clock whoever feeds it; fed by plain
 //       stores of the consumers it also holds up their shared-memory loads, the TMA unit reads
 //       shared memory on its own path;
+//   warp NC+3 (publisher): with all layers in one launch, makes the finished tiles known to the other
+//       SMs (a.tile_done).  That takes fences, and a fence lasts thousands of cycles while the SM's
+//       stores are in flight; here they delay nobody and cover several items at once;
 //   warps 0..NC-1 (consumers): warp (ms, sg) keeps a TM x 8 register tile per lane
 //       (columns m' = tile + ms*32*TM + j*32 + lane, strategies sg*8 .. sg*8+7), waits for the
 //       stage, runs one fused add-min per relaxation, releases the stage, and after the last
@@ -327,15 +338,17 @@ __device__ __forceinline__ ItemPos item_at(long long item, int nt, int nsb) {
     return p;
 }
 
-// Item records in flight: the producer runs at most (stages + 3) items ahead of the store warp.
-constexpr int kDescRing = 16;
+// Item records in flight: the producer runs at most (stages + 3) items ahead of the store warp, and
+// the store warp at most kPublishLag items ahead of the publisher.
+constexpr int kPublishLag = 8;
+constexpr int kDescRing = 32;
 
 // Shared memory: NST stages of [KS][TMB] previous-layer values + [KS][SB] trans values, then per
 // stage a small record the producer fills for the item whose last chunk sits in that stage:
 // mem(l,s) and time(l,s) of the s-block and the instance index; then the staging tile of the
 // outputs and its header.
 template <int TM, int NSG, int NMS, bool ARG, bool MULTI>
-__global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
+__global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
                                                                               const __grid_constant__ CUtensorMap map_t)
 {
@@ -355,6 +368,8 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
     __shared__ int fill_count;                             // helper -> store warp: first tiles whose unreachable cells are written
     __shared__ int4 desc[kDescRing];                       // item records: layer (-1: no more items), instance, tile, s-block
     __shared__ int desc_count;                             // records posted so far
+    __shared__ int drained_count, published_count;         // store warp -> publisher: items whose stores are complete; and back
+    __shared__ int store_exit;                             // the store warp has left
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
@@ -382,6 +397,9 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         mbar_init(&out_empty, 1);
         fill_count = 0;
         desc_count = 0;
+        drained_count = 0;
+        published_count = 0;
+        store_exit = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -399,22 +417,31 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         // this launch's items are g_base .. g_end-1 of the sequence over all layers
         const long long g_base = a.istart[l_first], g_end = a.istart[l_last];
         unsigned long long* const work = a.work + (MULTI ? 0 : l_first);
-        int l = l_first, nt = a.ntiles[l_first];          // layer of the item at hand (items arrive in increasing order)
+        // Global loads and atomics come back after thousands of cycles while the SM's stores are in
+        // flight, so the next item is taken and decoded in the shadow of this item's waits.
+        int nl = l_first, nt = a.ntiles[l_first], ntp = a.ntiles[l_first - 1];   // decoder state: layer, its tiles, the tiles of the layer before
         long long lbeg = g_base, lend = a.istart[l_first + 1];
-        for (int it = 0;; ++it) {
-            long long g = 0;
-            if (lane == 0) g = g_base + (long long)atomicAdd(work, 1ull);
-            g = __shfl_sync(0xffffffffu, g, 0);
-            const bool last = g >= g_end;
-            ItemPos pos = {0, 0, 0};
-            int i = 0;
-            if (!last) {
-                while (g >= lend) { ++l; lbeg = lend; lend = a.istart[l + 1]; nt = a.ntiles[l]; }
-                pos = item_at(g - lbeg, nt, pl.nsb);
-                i = a.order[pos.oi];
+        struct Item { int l, i, mt, sb, ntp; };
+        auto grab = [&]() -> long long {                  // lane 0 holds the result
+            return lane == 0 ? g_base + (long long)atomicAdd(work, 1ull) : 0;
+        };
+        auto decode = [&](long long g0) -> Item {          // items arrive in increasing order
+            const long long g = __shfl_sync(0xffffffffu, g0, 0);
+            Item r = {-1, 0, 0, 0, 0};
+            if (g < g_end) {
+                while (g >= lend) { ++nl; lbeg = lend; lend = a.istart[nl + 1]; ntp = nt; nt = a.ntiles[nl]; }
+                const ItemPos p = item_at(g - lbeg, nt, pl.nsb);
+                r.l = nl; r.i = a.order[p.oi]; r.mt = p.mt; r.sb = p.sb; r.ntp = ntp;
             }
+            return r;
+        };
+        Item cur = decode(grab());
+        for (int it = 0;; ++it) {
+            const int l = cur.l, i = cur.i;
+            const bool last = l < 0;
+            const ItemPos pos = {0, cur.mt, cur.sb};
             if (lane == 0) {
-                desc[it % kDescRing] = make_int4(last ? -1 : l, i, pos.mt, pos.sb);
+                desc[it % kDescRing] = make_int4(l, i, pos.mt, pos.sb);
                 __threadfence_block();
                 *reinterpret_cast<volatile int*>(&desc_count) = it + 1;
             }
@@ -429,36 +456,39 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 if (lane == 0) mbar_arrive(&full_bar[st]);
                 return;
             }
+            const long long g_next = grab();              // lands while the dependencies are polled
             const int row0 = a.C ? (l - 1) * S : ((l - 1) & 1) * a.B * S;      // row of (instance 0, layer l-1, s'=0)
             const int m0 = pos.mt * TMB;
             if (MULTI && tile_done && l > 1) {
                 // bounded wait for the tiles of layer l-1 (all their s-blocks) this item reads
                 // = s-blocks x the layers up to l-1 that ran the tile (trailing tiles are left out layer by layer)
                 const int32_t* const ran = a.tcount + (size_t)(l - 1) * pl.ntiles_m;
-                // one lane per tile polls (relaxed), then one acquire fence for the warp
+                // One lane per tile polls with acquire loads; the warp barrier below orders them before
+                // lane 0's TMA loads.  The writes the counters stand for were pushed through the publisher's
+                // proxy fence before its release, so no fence is needed here (it would cost this warp
+                // thousands of cycles per item while the SM's own stores are in flight).
                 bool ok = true;
-                const int tlast = min(pos.mt, a.ntiles[l - 1] - 1);      // tiles the previous layer did not run store nothing
+                const int tlast = min(pos.mt, cur.ntp - 1);              // tiles the previous layer did not run store nothing
                 for (int t0 = max(0, pos.mt - kdep); t0 <= tlast && ok; t0 += 32) {
                     const int t = t0 + lane;
                     if (t <= tlast) {
                         const int32_t* c = tile_done + (size_t)i * pl.ntiles_m + t;
                         WaitClock wc;
                         const int need = ran[t] * pl.nsb;
-                        while (ld_relaxed_gpu(c) < need) {
+                        while (ld_acquire_gpu(c) < need) {
                             if (wc.expired()) { ok = false; break; }
-                            __nanosleep(64);
+                            __nanosleep(200);
                         }
                     }
                     ok = __all_sync(0xffffffffu, ok);
                 }
-                __threadfence();                                         // acquire: the tiles' data is ordered after the counters
-                asm volatile("fence.proxy.async;" ::: "memory");         // ... and visible to the TMA loads below
                 __syncwarp();
                 if (!ok) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
             }
+            const Item nxt = decode(g_next);              // its instance index lands while this item's stages are awaited
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
             const int yc = row0 + i * inst_rows;
@@ -500,11 +530,12 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                 }
                 __syncwarp();
             }
+            cur = nxt;
         }
     }
     if (warp == NC + 1) {
         // ------------------------------------------------------------ helper
-        int n = 0;
+        int n = 0, nfilled = 0;
         for (int it = 0;; ++it) {
             {
                 WaitClock wc;                             // the producer posts the item's record
@@ -513,7 +544,7 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                         if (lane == 0) atomicExch(a.err, 1);
                         return;
                     }
-                    __nanosleep(32);
+                    __nanosleep(200);
                 }
                 __threadfence_block();
             }
@@ -569,10 +600,13 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                     }
                 }
                 if (MULTI && tile_done) {
-                    // the store warp publishes the tile; it must know these cells are out
-                    __threadfence();
+                    // The tile is published only after these cells: the count goes to the store warp and
+                    // on to the publisher by release / acquire in shared memory, and the publisher's fence
+                    // is cumulative.  (A fence here would hold this warp, and with it the records of the
+                    // next items, for thousands of cycles.)  A counter, not a barrier phase: this warp may
+                    // be several first tiles ahead.
                     __syncwarp();
-                    if (lane == 0) atomicAdd(&fill_count, 1);      // a counter, not a barrier phase: the helper may be several first tiles ahead
+                    if (lane == 0) st_release_cta(&fill_count, ++nfilled);
                 }
             }
         }
@@ -585,22 +619,20 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
         // table columns above M do not exist.  Each lane takes rows lane, lane+32: the 16-byte aligned
         // middle leaves as one bulk store, the few cells before and after it as plain stores.
         int it = 0;
-        int32_t* unpublished = nullptr;                   // tile counter of the previous item, not yet bumped
         int nfill = 0;                                    // first tiles seen so far
-        // Publishing a tile: its bulk stores complete, every lane's plain stores fenced, one release add.
-        auto publish = [&](int32_t* counter) {
-            __threadfence();
+        const bool publishing = MULTI && tile_done;
+        // every way out tells the publisher (after the last hand-over, in program order)
+        auto leave = [&](bool failed) {
+            if (failed && lane == 0) atomicExch(a.err, 1);
             __syncwarp();
-            if (lane == 0) {
-                asm volatile("fence.proxy.async;" ::: "memory");
-                red_release_gpu_add(counter, 1);
-            }
+            if (lane == 0) *reinterpret_cast<volatile int*>(&store_exit) = 1;
         };
         for (;; ++it) {
-            if (!mbar_wait(&out_full, it & 1)) {
-                if (lane == 0) atomicExch(a.err, 1);
-                return;
-            }
+            if (!mbar_wait(&out_full, it & 1)) { leave(true); return; }
+            // The consumers' staging writes (generic proxy) are ordered before this point by the barrier;
+            // one proxy fence here makes them visible to the bulk stores below.  In the consumers it would
+            // stall sixteen warps while the producer's loads are in flight.
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             const int4 d = desc[it % kDescRing];
             const int l = d.x, i = d.y;
             if (l < 0) break;                                     // no more items
@@ -627,36 +659,69 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
             bulk_wait_read();                                     // the staging tile may be overwritten
             __syncwarp();
             if (lane == 0) mbar_arrive(&out_empty);
-            if (MULTI && tile_done) {
-                // The previous item's bulk stores were issued a whole item ago: waiting for all groups
-                // but the newest costs nothing, and then that item is published.
-                int32_t* mine = tile_done + (size_t)i * pl.ntiles_m + pos.mt;
+            if (publishing) {
+                // Hand the item to the publisher warp once its stores are complete.  Making them visible
+                // to the other SMs takes a fence, and a fence takes thousands of cycles while stores are
+                // in flight: this warp must be back for the next tile sooner than that.
                 if (pos.mt == 0) {                                // the helper's fill of this tile (it runs ahead)
                     ++nfill;
                     WaitClock wc;
-                    while (*reinterpret_cast<volatile int*>(&fill_count) < nfill) {
-                        if (wc.expired()) {
-                            if (lane == 0) atomicExch(a.err, 1);
-                            return;
-                        }
-                        __nanosleep(64);
+                    while (ld_acquire_cta(&fill_count) < nfill) {
+                        if (wc.expired()) { leave(true); return; }
+                        __nanosleep(200);
                     }
                 }
-                if (unpublished) { bulk_wait_all_but_last(); publish(unpublished); }
-                // Deferred only when this CTA's next item is known and sits in the same layer, so that
-                // it cannot itself be waiting for this tile; near a layer's end the tile is published at once.
-                bool defer = false;
-                if (*reinterpret_cast<volatile int*>(&desc_count) > it + 1) {
-                    __threadfence_block();
-                    defer = desc[(it + 1) % kDescRing].x == l;
+                bulk_wait_all();
+                {
+                    WaitClock wc;                                 // the publisher reads item records: keep it close
+                    while (it + 1 - *reinterpret_cast<volatile int*>(&published_count) > kPublishLag) {
+                        if (wc.expired()) { leave(true); return; }
+                        __nanosleep(200);
+                    }
                 }
-                if (defer) unpublished = mine;
-                else { bulk_wait_all(); publish(mine); unpublished = nullptr; }
+                __syncwarp();                                     // every lane's plain stores before lane 0's release
+                if (lane == 0) st_release_cta(&drained_count, it + 1);
             }
         }
         bulk_wait_all();
-        if (unpublished) publish(unpublished);
+        leave(false);
         return;
+    }
+
+    if (warp == NC + 3) {
+        // ------------------------------------------------------------ publisher
+        // Publishes finished tiles in a.tile_done: one proxy fence and one release fence for all the
+        // items the store warp has handed over since the last round, then one relaxed add per item.
+        // The hand-over (release / acquire in shared memory) puts the store warp's and the helper's
+        // writes before the fence, which is cumulative.
+        if (!(MULTI && tile_done)) return;
+        int published = 0;
+        for (;;) {
+            int drained = 0, fin = 0;
+            WaitClock wc;
+            for (;;) {
+                fin = *reinterpret_cast<volatile int*>(&store_exit);      // read before the count: then the count is final
+                drained = ld_acquire_cta(&drained_count);
+                if (drained > published || fin) break;
+                if (wc.expired()) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+                __nanosleep(400);
+            }
+            if (drained == published) return;                     // the store warp has left and nothing is pending
+            if (lane == 0) {
+                asm volatile("fence.proxy.async;" ::: "memory");  // the data is read by other SMs' TMA loads
+                __threadfence();
+                for (int k = published; k < drained; ++k) {
+                    const int4 d = desc[k % kDescRing];
+                    red_relaxed_gpu_add(tile_done + (size_t)d.y * pl.ntiles_m + d.z, 1);
+                }
+                *reinterpret_cast<volatile int*>(&published_count) = drained;
+            }
+            __syncwarp();
+            published = drained;
+        }
     }
 
     // ---------------------------------------------------------------- consumers
@@ -821,9 +886,8 @@ __global__ void __launch_bounds__((NSG * NMS + 3) * 32, 1) layer_tiled_kernel(co
                     }
             }
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // staging writes -> visible to the TMA unit
         __syncwarp();
-        if (lane == 0) mbar_arrive(&out_full);
+        if (lane == 0) mbar_arrive(&out_full);                // release: the staging writes come before it
     }
 }
 
@@ -864,9 +928,9 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
     }
     if (l_last - l_first > 1) {
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[0], (void*)&maps[1]};
-        return cudaLaunchCooperativeKernel((const void*)kern_multi, dim3(pl.grid), dim3((NSG * NMS + 3) * 32), args, (size_t)pl.smem, st);
+        return cudaLaunchCooperativeKernel((const void*)kern_multi, dim3(pl.grid), dim3((NSG * NMS + 4) * 32), args, (size_t)pl.smem, st);
     }
-    kern<<<pl.grid, (NSG * NMS + 3) * 32, pl.smem, st>>>(a, pl, l_first, l_last, maps[0], maps[1]);
+    kern<<<pl.grid, (NSG * NMS + 4) * 32, pl.smem, st>>>(a, pl, l_first, l_last, maps[0], maps[1]);
     return cudaGetLastError();
 }
 
@@ -928,7 +992,7 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     pl->nms = 16 / pl->nsg;
     if (pl->nms < 1) pl->nms = 1;
     pl->tmb = pl->nms * 32 * pl->tm;
-    pl->threads = (pl->nsg * pl->nms + 3) * 32;           // consumer warps + producer + helper + store warp
+    pl->threads = (pl->nsg * pl->nms + 4) * 32;           // consumer warps + producer, helper, store and publisher warps
     // stages of ks * (tmb + sb) ints: aim at <= 40 KB each, 2..4 of them in the opt-in shared memory
     const int extra = ((kMaxStages * (2 * pl->sb + 4) + 31) & ~31) * 4      // item records
                       + (pl->sb * (pl->tmb + 4) + pl->sb + 4) * 4;        // staging tile and its header
@@ -942,7 +1006,7 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
         if (ks >= 8) ks = (ks + 7) & ~7;
         stage_bytes = (ks * row + 127) & ~127;
         nst = avail / stage_bytes;
-        if (nst >= 2 || ks == 1) break;
+        if (nst >= (getenv("GALV_MIN_STAGES") ? atoi(getenv("GALV_MIN_STAGES")) : 2) || ks == 1) break;
     }
     if (nst > kMaxStages) nst = kMaxStages;
     if (nst < 2) return false;

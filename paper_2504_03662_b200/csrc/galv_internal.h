@@ -30,7 +30,7 @@ struct DpPlan {
     int nst;       // pipeline stages in shared memory
     int tma_t;     // trans rows are 16-byte aligned: staged by a tiled TMA box, else by plain copies
     int ntiles_m;  // ceil((M+1) / tmb)
-    int threads;   // (nsg * nms + 3) * 32: consumer warps, producer warp, helper warp, store warp
+    int threads;   // (nsg * nms + 4) * 32: consumer warps, producer, helper, store and publisher warps
     int smem;      // dynamic shared memory bytes
     int grid;      // resident CTAs
 };

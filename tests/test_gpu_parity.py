@@ -293,6 +293,19 @@ def test_alu_probe_runs(galv):
     assert all(1e11 < r < 1e15 for r in rates), rates
 
 
+@pytest.mark.parametrize("flags", [1, 1 | 1024, 1 | 512, 3])
+def test_layers_with_different_tile_counts(orc, galv, flags):
+    """One heavy layer leaves its trailing tiles out; the layers after it run them again.
+
+    With all layers in one launch an item waits for the tiles of the layer before; how far a tile's
+    counter has to be depends on how many earlier layers ran that tile at all.
+    """
+    w = inputs.random_tables(41, 3, 7, 64, 1500, mem_lo=1, mem_hi=60, time_hi=3000)
+    w.mem_q[:, 2, :] += 800                      # layer 2: nothing lands above column 1500 - 801
+    w.mem_q[:, 5, :] += 300
+    check_batch(orc, galv, w, flags)
+
+
 @pytest.mark.parametrize("flags", [1, 1 | 512])
 def test_bounded_waits_run_out_cleanly(orc, galv, flags):
     """A stage that never fills: the waits give up, the status says TIMEOUT, the context keeps working."""
