@@ -109,6 +109,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         if (wc.expired()) return false;
     return true;
 }
+// The same for the role warps, which wait long and often: a warp that spins on try_wait takes issue
+// slots and ALU cycles from the four consumer warps on its scheduler, so it sleeps between polls.
+__device__ __forceinline__ bool mbar_wait_idle(uint64_t* bar, uint32_t parity) {
+    WaitClock wc;
+    while (!mbar_try_wait(bar, parity)) {
+        if (wc.expired()) return false;
+        __nanosleep(100);
+    }
+    return true;
+}
 // 1-D bulk async copy global -> shared, completion counted in bytes on an mbarrier.
 // dst, src 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -449,7 +459,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             if (last) {
                 // the consumers learn it through a stage that carries no data
                 const int st = n % NST;
-                if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                if (n >= NST && !mbar_wait_idle(&empty_bar[st], ((n / NST) - 1) & 1)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
@@ -498,7 +508,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             const bool skip = a.front && m0 + TMB - 1 < a.front[(size_t)i * a.Lmax + (l - 1)];
             for (int kc = 0; kc < NKC; ++kc, ++n) {
                 const int st = n % NST;
-                if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                if (n >= NST && !mbar_wait_idle(&empty_bar[st], ((n / NST) - 1) & 1)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
@@ -553,7 +563,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             ItemPos pos = {0, d.z, d.w};
             if (l < 0) {
                 const int st = n % NST;
-                if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                if (n >= NST && !mbar_wait_idle(&empty_bar[st], ((n / NST) - 1) & 1)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
@@ -571,7 +581,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             const int tq1 = lane + 32 < sbw ? __ldg(a.time_q + qrow + lane + 32) : 0;
             for (int kc = 0; kc < NKC; ++kc, ++n) {
                 const int st = n % NST;
-                if (n >= NST && !mbar_wait(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                if (n >= NST && !mbar_wait_idle(&empty_bar[st], ((n / NST) - 1) & 1)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
@@ -628,7 +638,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             if (lane == 0) *reinterpret_cast<volatile int*>(&store_exit) = 1;
         };
         for (;; ++it) {
-            if (!mbar_wait(&out_full, it & 1)) { leave(true); return; }
+            if (!mbar_wait_idle(&out_full, it & 1)) { leave(true); return; }
             // The consumers' staging writes (generic proxy) are ordered before this point by the barrier;
             // one proxy fence here makes them visible to the bulk stores below.  In the consumers it would
             // stall sixteen warps while the producer's loads are in flight.
@@ -867,10 +877,11 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                     if (j < nj) R[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
             }
             if (ms == 0) {
+                // lane u posts mem of strategy u: selects and one store (eight divergent stores cost a thousand cycles)
+                int v = mm[0];
 #pragma unroll
-                for (int u = 0; u < TS; ++u)
-                    if (lane == u) hdr0[s0l + u] = mm[u];
-                if (sg == 0 && lane == 0) hdr0[SB] = inst;
+                for (int u = 1; u < TS; ++u) v = lane == u ? mm[u] : v;
+                if (lane < TS) hdr0[s0l + lane] = v;
             }
             if (ARG && nj > 0) {
                 const int s0 = pos.sb * SB + s0l;
