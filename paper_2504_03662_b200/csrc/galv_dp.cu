@@ -330,7 +330,7 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 //       chunk adds time(l,s) and writes its tile into the staging tile, row s shifted by
 //       mem(l,s) mod 4 so that column m' + mem(l,s) of the table is 16-byte aligned with it.
 // Stages are handed over with mbarriers (full: bytes landed and record written; empty: every consumer
-// warp done; out_full / out_empty for the staging tile), so there is no block-wide barrier in the
+// warp done; out_full for the staging tile, a counter for its drain), so there is no block-wide barrier in the
 // loop.  Every wait is bounded; a wait that runs out sets the error flag and the role returns.
 
 constexpr int kMaxStages = 4;
@@ -374,7 +374,9 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
-    __shared__ __align__(8) uint64_t out_full, out_empty;  // staging tile written / drained
+    __shared__ __align__(8) uint64_t out_full;             // staging tile written (all consumer warps)
+    __shared__ int out_drained;                            // items whose staging tile the store warp has read out: a plain
+                                                           // counter, its acquire load returns ten times sooner than a barrier wait
     __shared__ int fill_count;                             // helper -> store warp: first tiles whose unreachable cells are written
     __shared__ int4 desc[kDescRing];                       // item records: layer (-1: no more items), instance, tile, s-block
     __shared__ int desc_count;                             // records posted so far
@@ -404,7 +406,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     if (tid == 0) {
         for (int k = 0; k < NST; ++k) { mbar_init(&full_bar[k], 2); mbar_init(&empty_bar[k], NC); }
         mbar_init(&out_full, NC);
-        mbar_init(&out_empty, 1);
+        out_drained = 0;
         fill_count = 0;
         desc_count = 0;
         drained_count = 0;
@@ -668,7 +670,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             bulk_commit();
             bulk_wait_read();                                     // the staging tile may be overwritten
             __syncwarp();
-            if (lane == 0) mbar_arrive(&out_empty);
+            if (lane == 0) st_release_cta(&out_drained, it + 1);
             if (publishing) {
                 // Hand the item to the publisher warp once its stores are complete.  Making them visible
                 // to the other SMs takes a fence, and a fence takes thousands of cycles while stores are
@@ -739,7 +741,15 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     int acc[TM][TS];
     int arg[ARG ? TM : 1][ARG ? TS : 1];
     (void)arg;
-    int n = 0;
+    int n = 0, cst = 0;
+    uint32_t cph = 0;
+    // bounded wait until the store warp has read items 0 .. upto-1 out of the staging tile
+    auto drained_wait = [&](int upto) -> bool {
+        WaitClock wc;
+        while (ld_acquire_cta(&out_drained) < upto)
+            if (wc.expired()) return false;
+        return true;
+    };
     for (int it = 0;; ++it) {
         int l = 0, mw = 0, nj = 0;
         ItemPos pos = {0, 0, 0};
@@ -752,8 +762,8 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             }
         int mm[TS], tt[TS], inst = 0;
         for (int kc = 0; kc < NKC; ++kc, ++n) {
-            const int st = n % NST;
-            if (!mbar_wait(&full_bar[st], (n / NST) & 1)) {
+            const int st = cst;                             // = n % NST, phase cph = (n / NST) & 1
+            if (!mbar_wait(&full_bar[st], cph)) {
                 if (lane == 0) atomicExch(a.err, 1);
                 return;
             }
@@ -764,7 +774,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                 if (l < 0) {
                     // no more items: wake the store warp and leave.  Not before it has taken the previous
                     // item: two completions of out_full in a row would hide the first from its parity wait.
-                    if (it > 0 && !mbar_wait(&out_empty, (it - 1) & 1)) {
+                    if (!drained_wait(it)) {
                         if (lane == 0) atomicExch(a.err, 1);
                         return;
                     }
@@ -857,11 +867,12 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);      // this warp is done reading the stage
+            if (++cst == NST) { cst = 0; cph ^= 1; }
         }
 
         // Epilogue: add time(l,s) and hand the tile to the store warps through the staging tile;
         // row s is written shifted by mem(l,s) mod 4 (see the store warps).
-        if (it > 0 && !mbar_wait(&out_empty, (it - 1) & 1)) {    // the previous item has been drained
+        if (!drained_wait(it)) {                             // the previous item has been drained
             if (lane == 0) atomicExch(a.err, 1);
             return;
         }
