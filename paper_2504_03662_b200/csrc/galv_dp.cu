@@ -24,6 +24,7 @@
 #include <cuda.h>
 
 #include <cstring>
+#include <type_traits>
 #include <cstdlib>
 
 #include "galv_internal.h"
@@ -369,6 +370,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     constexpr int NBOX = TMB / BOXC;
     constexpr int META = 2 * SB + 4;
     constexpr int RS = TMB + 4;                           // staging row: TMB columns + room for the shift
+    constexpr int KU = ARG ? 4 : 16;                      // k-steps per trip of the inner loop
     static_assert(TMB % BOXC == 0 && BOXC % (32 * TM) == 0, "a warp's columns must sit inside one box");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -795,47 +797,39 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             const int32_t* cs = stage0 + st * stage_elems + ((ms * (32 * TM)) / BOXC) * (KS * BOXC) + (ms * (32 * TM)) % BOXC + lane;
             const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
             if (nj == TM) {
+                // trips of KU k-steps, then of 4, then single ones: loop control and pointer bumps are ALU
+                // instructions too, one trip of 16 k-steps spends 4 of them on 512 relaxations
                 int k = 0;
-                for (; k + 4 <= kn; k += 4) {
+                auto steps = [&](auto ku) {
+                    constexpr int K = decltype(ku)::value;
+                    for (; k + K <= kn; k += K) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        int c[TM];
+                        for (int kk = 0; kk < K; ++kk) {
+                            int c[TM];
 #pragma unroll
-                        for (int j = 0; j < TM; ++j) c[j] = cs[kk * BOXC + j * 32];
-                        const int4 t0 = *reinterpret_cast<const int4*>(ts + kk * SB);
-                        const int4 t1 = *reinterpret_cast<const int4*>(ts + kk * SB + 4);
-                        const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+                            for (int j = 0; j < TM; ++j) c[j] = cs[kk * BOXC + j * 32];
+                            const int4 t0 = *reinterpret_cast<const int4*>(ts + kk * SB);
+                            const int4 t1 = *reinterpret_cast<const int4*>(ts + kk * SB + 4);
+                            const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
 #pragma unroll
-                        for (int j = 0; j < TM; ++j)
+                            for (int j = 0; j < TM; ++j)
 #pragma unroll
-                            for (int u = 0; u < TS; ++u) {
-                                if (ARG) {
-                                    const int cand = c[j] + t[u];
-                                    if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k + kk; }
-                                } else {
-                                    acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                                for (int u = 0; u < TS; ++u) {
+                                    if (ARG) {
+                                        const int cand = c[j] + t[u];
+                                        if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k + kk; }
+                                    } else {
+                                        acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                                    }
                                 }
-                            }
-                    }
-                    cs += 4 * BOXC;
-                    ts += 4 * SB;
-                }
-                for (; k < kn; ++k) {
-                    const int4 t0 = *reinterpret_cast<const int4*>(ts);
-                    const int4 t1 = *reinterpret_cast<const int4*>(ts + 4);
-                    const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-#pragma unroll
-                    for (int j = 0; j < TM; ++j) {
-                        const int c = cs[j * 32];
-#pragma unroll
-                        for (int u = 0; u < TS; ++u) {
-                            const int cand = c + t[u];
-                            if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
                         }
+                        cs += K * BOXC;
+                        ts += K * SB;
                     }
-                    cs += BOXC;
-                    ts += SB;
-                }
+                };
+                steps(std::integral_constant<int, KU>());
+                steps(std::integral_constant<int, 4>());
+                steps(std::integral_constant<int, 1>());
             } else if (nj > 0) {
                 // ragged last tile: only the first nj column groups carry work
                 for (int k = 0; k < kn; ++k) {
