@@ -335,6 +335,7 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 // loop.  Every wait is bounded; a wait that runs out sets the error flag and the role returns.
 
 constexpr int kMaxStages = 4;
+constexpr int kStaticSmemReserve = 512;                // the kernel's static shared memory (barriers, item ring, counters), rounded up
 
 struct ItemPos { int oi, mt, sb; };
 
@@ -351,8 +352,8 @@ __device__ __forceinline__ ItemPos item_at(long long item, int nt, int nsb) {
 
 // Item records in flight: the producer runs at most (stages + 3) items ahead of the store warp, and
 // the store warp at most kPublishLag items ahead of the publisher.
-constexpr int kPublishLag = 8;
-constexpr int kDescRing = 32;
+constexpr int kPublishLag = 5;
+constexpr int kDescRing = 16;
 
 // Shared memory: NST stages of [KS][TMB] previous-layer values + [KS][SB] trans values, then per
 // stage a small record the producer fills for the item whose last chunk sits in that stage:
@@ -1010,21 +1011,22 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     pl->tmb = pl->nms * 32 * pl->tm;
     pl->threads = (pl->nsg * pl->nms + 4) * 32;           // consumer warps + producer, helper, store and publisher warps
     // stages of ks * (tmb + sb) ints: aim at <= 40 KB each, 2..4 of them in the opt-in shared memory
-    const int extra = ((kMaxStages * (2 * pl->sb + 4) + 31) & ~31) * 4      // item records
-                      + (pl->sb * (pl->tmb + 4) + pl->sb + 4) * 4;        // staging tile and its header
-    const int avail = ctx->smem_optin - 2048 - extra;
+    const int staging = (pl->sb * (pl->tmb + 4) + pl->sb) * 4;              // staging tile and its header
+    const int budget = ctx->smem_optin - kStaticSmemReserve;               // dynamic shared memory a CTA may have
     const int row = (pl->tmb + pl->sb) * 4;
     // chunks of s': as few per item as leave room for two stages (every chunk costs the consumers
-    // a barrier hand-over), of equal size, multiples of 8 rows
-    int nkc = 1, ks = S, stage_bytes = 0, nst = 0;
+    // a barrier hand-over), of equal size, multiples of 8 rows; then as many stages as fit
+    int nkc = 1, ks = S, stage_bytes = 0, nst = 0, extra = 0;
     for (;; ++nkc) {
         ks = (S + nkc - 1) / nkc;
         if (ks >= 8) ks = (ks + 7) & ~7;
         stage_bytes = (ks * row + 127) & ~127;
-        nst = avail / stage_bytes;
-        if (nst >= (getenv("GALV_MIN_STAGES") ? atoi(getenv("GALV_MIN_STAGES")) : 2) || ks == 1) break;
+        for (nst = kMaxStages; nst >= 2; --nst) {
+            extra = ((nst * (2 * pl->sb + 4) + 31) & ~31) * 4 + staging;  // item records of the stages
+            if (nst * stage_bytes + extra <= budget) break;
+        }
+        if (nst >= 2 || ks == 1) break;
     }
-    if (nst > kMaxStages) nst = kMaxStages;
     if (nst < 2) return false;
     pl->ks = ks;
     pl->nst = nst;
@@ -1063,7 +1065,7 @@ cudaError_t galv_dp_configure(const galv_ctx* ctx)
     // opt every instantiation into the large dynamic shared memory once per context
     DpArgs a{};
     DpPlan pl{};
-    pl.smem = ctx->smem_optin - 2048;
+    pl.smem = ctx->smem_optin - kStaticSmemReserve;
     for (int nsg = 1; nsg <= 8; ++nsg) {
         pl.nsg = nsg;
         cudaError_t e = launch_tiled<false>(a, pl, 0, 0, nullptr, nullptr);
