@@ -40,7 +40,7 @@ ALU_PEAK_GOPS = 148 * 64 * 1.965
 # DRAM bytes (read + write) per LAYER of the layer_tiled_kernel, from the committed ncu captures under
 # profiles/ (captured on the first layers of the same batch: the kernel's traffic grows in proportion
 # to the layers a launch covers, so a launch over Lmax-1 layers moves (Lmax-1) times this).
-NCU_TRAFFIC_BYTES_PER_LAYER = {"config3_heterogeneous": 533.3e6, "config4_research_sweep": 541.4e6}
+NCU_TRAFFIC_BYTES_PER_LAYER = {"config3_heterogeneous": 534.0e6, "config4_research_sweep": 541.4e6}
 
 
 def workload_for(k: int, rank: int = 0, batch: int = 0, layers: int = 0):
@@ -181,6 +181,29 @@ def time_steps(torch, fn, steps, warmup, barrier):
     return e0.elapsed_time(e1) * 1e-3
 
 
+def cost_model_scaled(torch, galv, hbm_gbs, barrier, copies=8192):
+    """The cost-model kernels alone on `copies` instances of the heterogeneous stack: large enough to be
+    bandwidth-bound (the benchmark's own batch is launch-latency-bound).  Bytes counted: the int32 outputs."""
+    import numpy as np
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import _dev_bytes
+    w = inputs.config3(B=copies)
+    dev = torch.device("cuda", galv.device)
+    shape = gb.make_shape(w.B, w.Lmax, w.S, w.M, 0)
+    L = torch.from_numpy(np.ascontiguousarray(w.L, np.int32)).to(dev)
+    layers, strat, inst = _dev_bytes(w.layers, dev), _dev_bytes(w.strat, dev), _dev_bytes(w.inst, dev)
+    tq = torch.empty(w.B, w.Lmax, w.S, dtype=torch.int32, device=dev)
+    mq = torch.empty_like(tq)
+    xq = torch.empty(w.B, w.S, w.S, dtype=torch.int32, device=dev)
+    status = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    stride = 0 if w.layers.shape[0] == 1 else w.Lmax
+    fn = lambda: galv.galv_eval_costs(shape, L, layers, stride, strat, inst, None, None, tq, mq, xq, status)
+    t = time_steps(torch, fn, 10, 3, barrier) / 10
+    nbytes = 4 * (2 * tq.numel() + xq.numel())
+    return {"instances": copies, "elements": tq.numel(), "ms": t * 1e3, "bytes_written": nbytes,
+            "gb_per_s": nbytes / t / 1e9, "frac_of_hbm": nbytes / t / 1e9 / hbm_gbs}
+
+
 def launches_per_step(w) -> int:
     # cost + trans kernels, validate + schedule + base layer, ONE cooperative launch over all layers,
     # copy-last + finalize, backtrack
@@ -190,14 +213,17 @@ def launches_per_step(w) -> int:
 def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):
     from paper_2504_03662_b200.search import SearchBuffers
     sb = SearchBuffers(galv, w, flags)
-    galv.galv_set_profiling(True)
-    t = time_steps(torch, sb.step, steps, warmup, barrier)
-    layer_ms = galv.galv_last_layer_loop_ms()                    # all layer launches of the last search, back to back
+    for _ in range(warmup):
+        sb.step()
+    galv.galv_set_profiling(True)                                # one event pair around the layer launches of every timed search
+    t = time_steps(torch, sb.step, steps, 0, barrier)
+    layer_ms, layer_min, layer_max, layer_n = galv.galv_layer_loop_ms_stats()   # mean over the timed searches (the last 64)
     galv.galv_set_profiling(False)
     res = sb.results()
     out = {"seconds": t, "ms_per_step": t / steps * 1e3, "cells_per_s": w.cells * steps / t,
            "relax_per_s": w.relaxations * steps / t, "searches_per_s": w.B * steps / t,
            "layer_kernel_ms_avg": layer_ms / max(1, w.Lmax - 1), "layer_loop_ms": layer_ms,
+           "layer_loop_ms_min": layer_min, "layer_loop_ms_max": layer_max, "layer_loop_launches_timed": layer_n,
            "feasible": int((res["status"] == 0).sum()), "opt_cost_sum": int(res["opt_cost"][res["status"] == 0].sum())}
     return sb, out
 
@@ -293,7 +319,8 @@ def main():
                      "algorithmic_bytes_per_launch": 2 * 4 * w.B * w.S * w.m_pitch * (w.Lmax - 1),
                      "algorithmic_ops_per_launch": relax_per_launch,
                      "kernel": "layer_tiled_kernel (one cooperative launch over all layers)",
-                     "launch_ms": r["layer_loop_ms"],
+                     "launch_ms": r["layer_loop_ms"], "launch_ms_min": r["layer_loop_ms_min"],
+                     "launch_ms_max": r["layer_loop_ms_max"], "launches_timed": r["layer_loop_launches_timed"],
                      "peak_source": "derived: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min per lane per clock"},
     }
 
@@ -348,6 +375,7 @@ def main():
             del sbk, g
             torch.cuda.empty_cache()
         line["others"] = others
+        line["cost_model_scaled"] = cost_model_scaled(torch, galv, hbm_gbs, barrier)
 
     if rank == 0 and world == 1 and not args.no_cpu:
         from oracle import oracle

@@ -325,10 +325,15 @@ int galv_probe_int_alu(galv_ctx* ctx, int kind, int iters, double* ops_per_s, vo
  * on, galv_dp_search records one CUDA event before its first layer launch and
  * one after its last; galv_last_layer_loop_ms waits for the second and returns
  * the milliseconds between them for the most recent search (host pointer).
- * Leave it off when capturing a CUDA graph.
+ * galv_layer_loop_ms_stats does the same for every search since profiling was
+ * switched on (the most recent 64 at most): mean, shortest and longest span in
+ * milliseconds and the number of searches they cover (host pointers).
+ * Switching profiling on or off forgets the spans.  Leave it off when capturing
+ * a CUDA graph.
  */
 int galv_set_profiling(galv_ctx* ctx, int on);
 int galv_last_layer_loop_ms(galv_ctx* ctx, float* ms);
+int galv_layer_loop_ms_stats(galv_ctx* ctx, float* mean_ms, float* min_ms, float* max_ms, int* searches);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,8 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgalv.so"
 
 EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "galv_eval_costs",
            "galv_dp_workspace_bytes", "galv_dp_search", "galv_backtrack", "galv_search_host_arena_bytes",
-           "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_dp_search_static", "galv_select_best", "galv_prune_strategies",
+           "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_layer_loop_ms_stats",
+           "galv_dp_search_static", "galv_select_best", "galv_prune_strategies",
            "galv_compact_tables", "galv_expand_plan", "galv_plan_cost", "galv_graph_create", "galv_graph_launch",
            "galv_graph_destroy", "galv_layer_optima", "galv_stage_partition")
 
@@ -82,6 +83,7 @@ def load_library() -> C.CDLL:
     lib.galv_probe_int_alu.argtypes = [vp, C.c_int, C.c_int, C.POINTER(C.c_double), vp]
     lib.galv_set_profiling.argtypes = [vp, C.c_int]
     lib.galv_last_layer_loop_ms.argtypes = [vp, C.POINTER(C.c_float)]
+    lib.galv_layer_loop_ms_stats.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int)]
     _lib = lib
     return lib
 
@@ -218,3 +220,9 @@ class Galv:
         out = C.c_float()
         self._check(self.lib.galv_last_layer_loop_ms(self.h, C.byref(out)))
         return out.value
+
+    def galv_layer_loop_ms_stats(self):
+        """(mean, min, max, searches) of the layer-launch spans since profiling was switched on."""
+        mean, lo, hi, n = C.c_float(), C.c_float(), C.c_float(), C.c_int()
+        self._check(self.lib.galv_layer_loop_ms_stats(self.h, C.byref(mean), C.byref(lo), C.byref(hi), C.byref(n)))
+        return mean.value, lo.value, hi.value, n.value

@@ -84,18 +84,18 @@ int galv_create(galv_ctx** out, int device_ordinal)
     ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
     ctx->err[0] = 0;
     ctx->profiling = 0;
-    ctx->ev_valid = 0;
-    ctx->ev0 = ctx->ev1 = nullptr;
+    ctx->prof_count = 0;
+    for (auto& ev : ctx->pev) ev = nullptr;
     int cur = -1;
     cudaGetDevice(&cur);
     if (cur != device_ordinal) cudaSetDevice(device_ordinal);
     e = galv_dp_configure(ctx);
-    if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev0);
-    if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev1);
+    for (auto& ev : ctx->pev)
+        if (e == cudaSuccess) e = cudaEventCreate(&ev);
     if (cur >= 0 && cur != device_ordinal) cudaSetDevice(cur);
     if (e != cudaSuccess) {
-        if (ctx->ev0) cudaEventDestroy(ctx->ev0);
-        if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+        for (auto& ev : ctx->pev)
+            if (ev) cudaEventDestroy(ev);
         delete ctx;
         return GALV_ERR_CUDA;
     }
@@ -105,10 +105,9 @@ int galv_create(galv_ctx** out, int device_ordinal)
 
 int galv_destroy(galv_ctx* ctx)
 {
-    if (ctx) {
-        if (ctx->ev0) cudaEventDestroy(ctx->ev0);
-        if (ctx->ev1) cudaEventDestroy(ctx->ev1);
-    }
+    if (ctx)
+        for (auto& ev : ctx->pev)
+            if (ev) cudaEventDestroy(ev);
     delete ctx;
     return GALV_OK;
 }
@@ -319,16 +318,39 @@ int galv_set_profiling(galv_ctx* ctx, int on)
 {
     if (!ctx) return GALV_ERR_INVALID_ARG;
     ctx->profiling = on != 0;
+    ctx->prof_count = 0;
     return GALV_OK;
 }
 
 int galv_last_layer_loop_ms(galv_ctx* ctx, float* ms)
 {
     if (!ctx || !ms) return GALV_ERR_INVALID_ARG;
-    if (!ctx->ev_valid) { set_err(ctx, "galv_last_layer_loop_ms: no profiled search yet"); return GALV_ERR_INVALID_ARG; }
-    cudaError_t e = cudaEventSynchronize(ctx->ev1);
-    if (e == cudaSuccess) e = cudaEventElapsedTime(ms, ctx->ev0, ctx->ev1);
+    if (ctx->prof_count < 1) { set_err(ctx, "galv_last_layer_loop_ms: no profiled search yet"); return GALV_ERR_INVALID_ARG; }
+    const int k = (ctx->prof_count - 1) % 64;
+    cudaError_t e = cudaEventSynchronize(ctx->pev[2 * k + 1]);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(ms, ctx->pev[2 * k], ctx->pev[2 * k + 1]);
     return e == cudaSuccess ? GALV_OK : cuda_fail(ctx, "galv_last_layer_loop_ms", e);
+}
+
+int galv_layer_loop_ms_stats(galv_ctx* ctx, float* mean_ms, float* min_ms, float* max_ms, int* searches)
+{
+    if (!ctx || !mean_ms || !min_ms || !max_ms || !searches) return GALV_ERR_INVALID_ARG;
+    if (ctx->prof_count < 1) { set_err(ctx, "galv_layer_loop_ms_stats: no profiled search yet"); return GALV_ERR_INVALID_ARG; }
+    const int n = ctx->prof_count < 64 ? ctx->prof_count : 64;
+    double sum = 0.0;
+    float lo = 0.f, hi = 0.f;
+    for (int j = 0; j < n; ++j) {
+        const int k = (ctx->prof_count - 1 - j) % 64;
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(ctx->pev[2 * k + 1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, ctx->pev[2 * k], ctx->pev[2 * k + 1]);
+        if (e != cudaSuccess) return cuda_fail(ctx, "galv_layer_loop_ms_stats", e);
+        sum += ms;
+        if (j == 0 || ms < lo) lo = ms;
+        if (j == 0 || ms > hi) hi = ms;
+    }
+    *mean_ms = (float)(sum / n); *min_ms = lo; *max_ms = hi; *searches = n;
+    return GALV_OK;
 }
 
 int galv_probe_int_alu(galv_ctx* ctx, int kind, int iters, double* ops_per_s, void* stream)

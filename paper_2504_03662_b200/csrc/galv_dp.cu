@@ -1134,7 +1134,8 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
         ap.tile_done = a.tile_done;
         if ((e = cudaMemsetAsync(a.tile_done, 0, (size_t)B * pl.ntiles_m * 4, st)) != cudaSuccess) return e;
     }
-    if (ctx->profiling) cudaEventRecord(ctx->ev0, st);
+    const int pk = ctx->prof_count % 64;
+    if (ctx->profiling) cudaEventRecord(ctx->pev[2 * pk], st);
     if (persistent) {
         if ((e = launch_tiled<false>(ap, pl, 1, Lmax, st, maps)) != cudaSuccess) return e;
     }
@@ -1148,7 +1149,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
         }
         if (e != cudaSuccess) return e;
     }
-    if (ctx->profiling) { cudaEventRecord(ctx->ev1, st); ctx->ev_valid = 1; }
+    if (ctx->profiling) { cudaEventRecord(ctx->pev[2 * pk + 1], st); ++ctx->prof_count; }
     for (int b0 = 0; b0 < B; b0 += 65535) {                   // grid.y limit
         DpArgs c = a;
         const int nb = (B - b0 < 65535) ? B - b0 : 65535;

@@ -11,9 +11,9 @@ struct galv_ctx {
     int device;
     int num_sms;
     int smem_optin;      // max dynamic shared memory per block (bytes)
-    int profiling;       // record ev0/ev1 around the layer launches
-    int ev_valid;        // ev0/ev1 have been recorded at least once
-    cudaEvent_t ev0, ev1;
+    int profiling;       // record an event pair around the layer launches of every search
+    int prof_count;      // searches profiled since profiling was switched on
+    cudaEvent_t pev[2 * 64];   // ring of event pairs: search k uses pev[2*(k%64)], pev[2*(k%64)+1]
     char err[512];
 };
 
