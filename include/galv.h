@@ -251,6 +251,28 @@ int galv_plan_cost(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
                    const int32_t* plan, int64_t* cost, int64_t* mem_total, void* stream);
 
 /*
+ * Plan switch (Sections 3-4: the running job is resharded when the selector finds a better plan;
+ * the paper gives no rule for when that pays, this is the reading taken).
+ * galv_add_switch_cost: time_out(i,l,s) = time_q(i,l,s) + trans_l(cur_plan[i][l], s) / horizon[i]
+ * (integer division; saturating at GALV_INF): resharding layer l from its current strategy to s
+ * is paid once and spread over horizon[i] >= 1 iterations (smaller values count as 1).  Entries
+ * of cur_plan outside 0..S-1 (no plan yet) and layers l >= L[i] add nothing.  With
+ * GALV_TRANS_PER_LAYER layer l uses matrix l (matrix 0 for layer 0).  Searching time_out instead
+ * of time_q weighs iteration time against the price of getting there.  time_out may not alias
+ * time_q.  cur_plan int32 [B][Lmax], horizon int32 [B], time_out int32 [B][Lmax][S]; device.
+ * galv_switch_decision: decision[i] = 1 when new_cost[i] * (1000 + hysteresis_permille) <
+ * cur_cost[i] * 1000, i.e. the new optimum beats staying by the margin; also 1 when the running
+ * plan no longer fits (cur_cost[i] < 0 or >= GALV_INF) and the new one does; 0 when new_status[i]
+ * != 0 or new_cost[i] >= GALV_INF.  cur_cost int64 [B] (as written by galv_plan_cost), new_cost,
+ * new_status, decision int32 [B]; device.  hysteresis_permille >= 0.
+ */
+int galv_add_switch_cost(galv_ctx* ctx, const galv_shape* shape, const int32_t* L, const int32_t* time_q,
+                         const int32_t* trans_q, const int32_t* cur_plan, const int32_t* horizon,
+                         int32_t* time_out, void* stream);
+int galv_switch_decision(galv_ctx* ctx, int32_t B, const int64_t* cur_cost, const int32_t* new_cost,
+                         const int32_t* new_status, int32_t hysteresis_permille, int32_t* decision, void* stream);
+
+/*
  * Re-search pipeline (Sections 3-4: the selector re-runs at intervals from fresh measurements).
  * galv_graph_create captures galv_eval_costs (when layers != NULL) -> galv_dp_search ->
  * galv_backtrack on the given device buffers into a CUDA graph; galv_graph_launch replays it on

@@ -392,3 +392,36 @@ void orc_stage_partition(int Lm, int P, const int32_t *range_opt, int32_t *cuts,
     free(f);
     free(g);
 }
+
+/* ------------------------------------------------------------------ plan switch
+ *
+ * Runtime adaptation (Sections 3 and 4 of the paper: the monitor re-evaluates, the optimiser
+ * proposes a plan, the manager reshards the running job).  The paper gives no rule for when a
+ * switch pays; the reading taken here:
+ *   - moving layer l from its current strategy c_l to s reshards that layer once, at the price the
+ *     cost model puts on that change of layout, trans_l(c_l, s); spread over `horizon` iterations
+ *     the price per iteration is trans_l(c_l, s) / horizon (integer division), added to time(l,s);
+ *     c_l < 0 (no plan yet) adds nothing; a horizon below 1 counts as 1; sums saturate at ORC_INF;
+ *   - the job switches when the new optimum, raised by hysteresis_permille / 1000, is still below
+ *     the cost of staying: new * (1000 + h) < cur * 1000.  A current plan that no longer fits
+ *     (cost >= ORC_INF) is left whenever the new one is feasible; an infeasible new plan never wins.
+ */
+void orc_add_switch_cost(int L, int S, const int32_t *time, const int32_t *trans, int64_t tl,
+                         const int32_t *cur_plan, int32_t horizon, int32_t *time_out)
+{
+    const int64_t H = horizon < 1 ? 1 : horizon;
+    for (int l = 0; l < L; l++)
+        for (int s = 0; s < S; s++) {
+            int64_t v = time[l * S + s];
+            const int c = cur_plan[l];
+            if (c >= 0 && c < S) v += (int64_t)trans[l * tl + c * S + s] / H;
+            time_out[l * S + s] = v >= ORC_INF ? ORC_INF : (int32_t)v;
+        }
+}
+
+int orc_switch_decision(int64_t cur_cost, int64_t new_cost, int32_t hysteresis_permille)
+{
+    if (new_cost >= ORC_INF) return 0;
+    if (cur_cost >= ORC_INF) return 1;
+    return new_cost * (1000 + (int64_t)hysteresis_permille) < cur_cost * 1000;
+}

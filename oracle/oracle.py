@@ -161,3 +161,16 @@ def stage_partition(range_opt, P: int):
     cuts = np.empty(P + 1, np.int32); bn = C.c_int32()
     lib().orc_stage_partition(Lm, P, pr, cuts.ctypes.data_as(C.c_void_p), C.byref(bn))
     return bn.value, cuts
+
+
+def add_switch_cost(time, trans, cur_plan, horizon: int):
+    """time'(l,s) = time(l,s) + trans_l(cur_plan[l], s) // horizon (see orc_add_switch_cost)."""
+    time, pt = _i32(time); trans, px = _i32(trans); cur, pc = _i32(cur_plan)
+    L, S = time.shape
+    out = np.empty((L, S), np.int32)
+    lib().orc_add_switch_cost(L, S, pt, px, _tl(trans, L, S), pc, int(horizon), out.ctypes.data_as(C.c_void_p))
+    return out
+
+
+def switch_decision(cur_cost: int, new_cost: int, hysteresis_permille: int) -> int:
+    return int(lib().orc_switch_decision(C.c_int64(int(cur_cost)), C.c_int64(int(new_cost)), int(hysteresis_permille)))

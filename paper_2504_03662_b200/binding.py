@@ -28,7 +28,8 @@ EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "g
            "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_layer_loop_ms_stats",
            "galv_dp_search_static", "galv_select_best", "galv_prune_strategies",
            "galv_compact_tables", "galv_expand_plan", "galv_plan_cost", "galv_graph_create", "galv_graph_launch",
-           "galv_graph_destroy", "galv_layer_optima", "galv_stage_partition")
+           "galv_graph_destroy", "galv_layer_optima", "galv_stage_partition", "galv_add_switch_cost",
+           "galv_switch_decision")
 
 
 class galv_shape(C.Structure):
@@ -72,6 +73,8 @@ def load_library() -> C.CDLL:
     lib.galv_compact_tables.argtypes = [vp, shp, C.c_int32] + [vp] * 8
     lib.galv_expand_plan.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, vp]
     lib.galv_plan_cost.argtypes = [vp, shp] + [vp] * 8
+    lib.galv_add_switch_cost.argtypes = [vp, shp] + [vp] * 7
+    lib.galv_switch_decision.argtypes = [vp, C.c_int32, vp, vp, vp, C.c_int32, vp, vp]
     lib.galv_graph_create.argtypes = [vp, shp, vp, vp, i64, vp, vp] + [vp] * 7 + [sz] + [vp] * 6 + [C.POINTER(vp)]
     lib.galv_graph_launch.argtypes = [vp, vp, vp]
     lib.galv_graph_destroy.argtypes = [vp]
@@ -169,6 +172,14 @@ class Galv:
     def galv_plan_cost(self, shape, L, time_q, mem_q, trans_q, plan, cost, mem_total):
         self._check(self.lib.galv_plan_cost(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),
                                             _ptr(plan), _ptr(cost), _ptr(mem_total), _stream()))
+
+    def galv_add_switch_cost(self, shape, L, time_q, trans_q, cur_plan, horizon, time_out):
+        self._check(self.lib.galv_add_switch_cost(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(trans_q), _ptr(cur_plan),
+                                                  _ptr(horizon), _ptr(time_out), _stream()))
+
+    def galv_switch_decision(self, B, cur_cost, new_cost, new_status, hysteresis_permille, decision):
+        self._check(self.lib.galv_switch_decision(self.h, B, _ptr(cur_cost), _ptr(new_cost), _ptr(new_status),
+                                                  int(hysteresis_permille), _ptr(decision), _stream()))
 
     def galv_graph_create(self, shape, L, layers, layer_stride_B, strat, inst, time_q, mem_q, trans_q, Ct, At, C_last,
                           workspace, budget, opt_cost, plan, mem_used, status, stream: int):
