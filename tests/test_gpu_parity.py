@@ -322,3 +322,40 @@ def test_bounded_waits_run_out_cleanly(orc, galv, flags):
     assert (bad.status.cpu().numpy() & gb.STATUS_TIMEOUT).all()
     # the same context and device then search normally
     check_batch(orc, galv, w, flags)
+
+
+@pytest.mark.parametrize("block", range(8))
+def test_one_launch_against_reference_kernel_on_many_shapes(galv, block):
+    """Consistency stress of the one-launch kernel (work queue, tile counters, role hand-overs): on random
+    shapes with many tiles, layers and ragged lengths its tables must equal those of the one-thread-per-cell
+    kernel, which the tests above tie to the oracle.  Run twice per shape: the second run reuses every buffer."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    rng = np.random.default_rng(1000 + block)
+    for case in range(10):
+        S = int(rng.choice([1, 5, 8, 24, 31, 32, 48, 64, 65, 100, 130, 256]))
+        Lmax = int(rng.integers(3, 30))
+        M = int(rng.integers(40, 5000))
+        pitch = (M + 32) // 32 * 32
+        B = int(max(1, min(rng.integers(1, 160), 3.0e8 // (Lmax * S * pitch * 4))))
+        mem_hi = int(rng.choice([3, M // 20 + 1, M // 3 + 1, 2 * M]))
+        w = inputs.random_tables(5000 + 100 * block + case, B, Lmax, S, M, ragged=bool(rng.integers(0, 2)),
+                                 mem_lo=int(rng.integers(0, 3)), mem_hi=mem_hi, trans_hi=int(rng.choice([0, 50, 50000])))
+        if rng.integers(0, 3) == 0:
+            w.mem_q[:, int(rng.integers(1, Lmax)), :] += M // 2       # one heavy layer: fewer tiles there
+        ref = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_REFERENCE)
+        ref.dp_search()
+        one = SearchBuffers(galv, w, gb.STORE_C_FULL | (gb.SKIP_INFEASIBLE if case % 3 == 2 else 0))
+        for _ in range(2):
+            one.C.fill_(-7)
+            one.dp_search()
+            torch.cuda.synchronize()
+            st = ref.status.cpu().numpy()
+            assert (one.status.cpu().numpy() == st).all(), (block, case)
+            for i in np.flatnonzero(st == 0):
+                Li = int(w.L[i])
+                assert torch.equal(one.C[i, :Li], ref.C[i, :Li]), (block, case, int(i), S, Lmax, M, B)
+            assert torch.equal(one.C_last[st == 0], ref.C_last[st == 0]), (block, case)
+        del ref, one
+        torch.cuda.empty_cache()
