@@ -204,25 +204,65 @@ __global__ void validate_kernel(int B, int Lmax, int S, int M, long long tl, con
     }
 }
 
-// Single CTA: nactive[l] = valid instances with L > l; order = valid instances, longest first.
+// Inclusive prefix sum of one value per thread over a block of 1024 threads; *total = the block's sum.
+__device__ long long block_scan_1024(long long v, long long* warp_sums, long long* total)
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const long long t = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += t;
+    }
+    if (lane == 31) warp_sums[wid] = v;
+    __syncthreads();
+    if (wid == 0) {
+        long long w = warp_sums[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const long long t = __shfl_up_sync(0xffffffffu, w, off);
+            if (lane >= off) w += t;
+        }
+        warp_sums[lane] = w;
+    }
+    __syncthreads();
+    if (wid > 0) v += warp_sums[wid - 1];
+    *total = warp_sums[31];
+    __syncthreads();
+    return v;
+}
+
+// Single CTA of 1024 threads: nactive[l] = valid instances with L > l; order = valid instances, longest first.
 // scratch = hist[Lmax+2] | fill[Lmax+2], zeroed by the host before the launch.
 // ntiles[l] = tiles of tmb columns per instance that can store anything in layer l: column m' lands at
 // m' + mem(l,s) <= M, so tiles starting above M - (smallest mem of the layer) are left out (at least one
 // tile stays: it also writes the cells no column maps to).
 // istart[l] = work items (instance, tile, s-block) of layers 1 .. l-1: the items of all layers in one sequence.
-__global__ void schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, int nsb, const int32_t* __restrict__ L,
+// tcount[l][t] = layers 1 .. l whose items include tile t.
+__global__ void __launch_bounds__(1024) schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, int nsb, const int32_t* __restrict__ L,
                                 const int32_t* __restrict__ status, int32_t* __restrict__ order, int32_t* __restrict__ nactive,
                                 int32_t* __restrict__ scratch, const int32_t* __restrict__ minmem_l, int32_t* __restrict__ ntiles,
                                 long long* __restrict__ istart, int32_t* __restrict__ tcount)
 {
+    __shared__ long long warp_sums[32];
     int32_t* hist = scratch;
     int32_t* fill = scratch + Lmax + 2;
     for (int i = threadIdx.x; i < B; i += blockDim.x)
         if (status[i] == 0) atomicAdd(&hist[L[i]], 1);
+    for (int l = threadIdx.x; l <= Lmax; l += blockDim.x) {
+        int nt = 1;
+        if (l < Lmax && minmem_l[l] <= M) nt = min(ntiles_m, (M - minmem_l[l]) / tmb + 1);
+        ntiles[l] = max(1, nt);
+    }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int run = 0;                                   // instances with L > l, from the top down
-        for (int l = Lmax; l >= 0; --l) { nactive[l] = run; run += hist[l]; }
+    {
+        long long carry = 0, total;                    // instances with L > l: a sum from the top layer down
+        for (int base = 0; base <= Lmax; base += 1024) {
+            const int l = Lmax - (base + (int)threadIdx.x);
+            const long long h = l >= 0 ? hist[l] : 0;
+            const long long incl = block_scan_1024(h, warp_sums, &total);
+            if (l >= 0) nactive[l] = (int32_t)(carry + incl - h);
+            carry += total;
+        }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < B; i += blockDim.x)
@@ -230,13 +270,6 @@ __global__ void schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, i
             const int Li = L[i];
             order[nactive[Li] + atomicAdd(&fill[Li], 1)] = i;   // instances longer than Li come first
         }
-    for (int l = threadIdx.x; l <= Lmax; l += blockDim.x) {
-        int nt = 1;
-        if (l < Lmax && minmem_l[l] <= M) nt = min(ntiles_m, (M - minmem_l[l]) / tmb + 1);
-        ntiles[l] = max(1, nt);
-    }
-    __syncthreads();
-    // tcount[l][t] = layers 1..l whose items include tile t
     for (int t = threadIdx.x; t < ntiles_m; t += blockDim.x) {
         int run = 0;
         tcount[t] = 0;
@@ -245,12 +278,15 @@ __global__ void schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, i
             tcount[(size_t)l * ntiles_m + t] = run;
         }
     }
-    if (threadIdx.x == 0) {
-        long long run = 0;
-        istart[0] = 0;
-        for (int l = 1; l <= Lmax; ++l) {
-            istart[l] = run;
-            if (l < Lmax) run += (long long)nactive[l] * ntiles[l] * nsb;
+    {
+        long long carry = 0, total;
+        if (threadIdx.x == 0) istart[0] = 0;
+        for (int base = 1; base <= Lmax; base += 1024) {
+            const int l = base + (int)threadIdx.x;
+            const long long v = l < Lmax ? (long long)nactive[l] * ntiles[l] * nsb : 0;
+            const long long incl = block_scan_1024(v, warp_sums, &total);
+            if (l <= Lmax) istart[l] = carry + incl - v;
+            carry += total;
         }
     }
 }

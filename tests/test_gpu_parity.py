@@ -359,3 +359,25 @@ def test_one_launch_against_reference_kernel_on_many_shapes(galv, block):
             assert torch.equal(one.C_last[st == 0], ref.C_last[st == 0]), (block, case)
         del ref, one
         torch.cuda.empty_cache()
+
+
+def test_kernel_span_statistics(galv):
+    """The timing hook keeps one event pair per profiled search and reports mean, shortest, longest."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    w = inputs.random_tables(3, 4, 6, 16, 700)
+    sb = SearchBuffers(galv, w, gb.STORE_C_FULL)
+    galv.galv_set_profiling(True)
+    with pytest.raises(gb.GalvError):
+        galv.galv_layer_loop_ms_stats()                      # nothing profiled yet
+    for _ in range(5):
+        sb.dp_search()
+    mean, lo, hi, n = galv.galv_layer_loop_ms_stats()
+    assert n == 5 and 0 < lo <= mean <= hi < 1000
+    assert lo <= galv.galv_last_layer_loop_ms() <= hi
+    for _ in range(70):                                      # more searches than pairs are kept
+        sb.dp_search()
+    assert galv.galv_layer_loop_ms_stats()[3] == 64
+    galv.galv_set_profiling(False)
+    torch.cuda.synchronize()
