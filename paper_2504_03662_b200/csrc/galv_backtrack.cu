@@ -76,28 +76,58 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, lon
     const int32_t* T0 = trans_q + (size_t)i * trans_inst;
     int m = bud;
     long long used = 0;
+    // One dependent memory round trip per layer: the cell's value is carried along (it is the chosen
+    // candidate of the step before), and the mem / time rows of the next layer down are fetched, whole,
+    // while this layer's candidates are in flight; lane k%32 keeps entries k, k+32, ... (S <= 256).
+    int cur = opt;                                             // C[l][m][s] of the cell the walk stands on
+    int mrow[8], trow[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int k = lane + 32 * j;
+        mrow[j] = k < S ? mq[(Li - 1) * S + k] : 0;
+        trow[j] = k < S ? tq[(Li - 1) * S + k] : 0;
+    }
     for (int l = Li - 1; l >= 0; --l) {
         if (lane == 0) pl[l] = s;
-        const int mm = mq[l * S + s];
+        int msel = mrow[0], tsel = trow[0];
+#pragma unroll
+        for (int j = 1; j < 8; ++j) {
+            msel = (s >> 5) == j ? mrow[j] : msel;
+            tsel = (s >> 5) == j ? trow[j] : tsel;
+        }
+        const int mm = __shfl_sync(0xffffffffu, msel, s & 31);
+        const int tt = __shfl_sync(0xffffffffu, tsel, s & 31);
         used += mm;
         if (l == 0) break;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {                          // rows of layer l-1, needed one step from now
+            const int k = lane + 32 * j;
+            mrow[j] = k < S ? mq[(l - 1) * S + k] : 0;
+            trow[j] = k < S ? tq[(l - 1) * S + k] : 0;
+        }
         int sp;
         if (A) {
             sp = A[((size_t)i * Lmax + l) * slice + (size_t)s * m_pitch + m];
         } else {
-            const int target = C[((size_t)i * Lmax + l) * slice + (size_t)s * m_pitch + m] - tq[l * S + s];
+            const int target = cur - tt;
             const int32_t* prev = C + ((size_t)i * Lmax + (l - 1)) * slice + (m - mm);
             const int32_t* T = T0 + (size_t)l * trans_layer;       // paid between layers l-1 and l
             sp = 255;
             for (int base = 0; base < S; base += 32) {
                 const int k = base + lane;
                 bool hit = false;
+                int c = kInf;
                 if (k < S) {
-                    const int c = prev[(size_t)k * m_pitch];
+                    c = prev[(size_t)k * m_pitch];
                     hit = (c < kInf) && (c + T[k * S + s] == target);
                 }
                 const unsigned b = __ballot_sync(0xffffffffu, hit);
-                if (b) { sp = base + __ffs(b) - 1; break; }
+                if (b) {
+                    const int src = __ffs(b) - 1;
+                    sp = base + src;
+                    cur = __shfl_sync(0xffffffffu, c, src);
+                    break;
+                }
             }
         }
         if (sp >= S) {                 // cannot happen on consistent tables; stop instead of walking off
