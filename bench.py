@@ -355,6 +355,16 @@ def main():
         line["opt_cost_sum"] = r["opt_cost_sum"]
         del sbs
         torch.cuda.empty_cache()
+        # Cost-only search: no table kept, two layers roll in the workspace (optimum per instance, no plan).
+        # All the relaxations are done; the tables' HBM footprint is 2 layers instead of Lmax.
+        sbc, rc = bench_workload(torch, galv, w, max(5, args.steps // 2), 3, barrier, flags=0)
+        line["cost_only"] = {"ms_per_step": rc["ms_per_step"], "cells_per_s": rc["cells_per_s"],
+                             "searches_per_s": rc["searches_per_s"], "opt_cost_sum": rc["opt_cost_sum"],
+                             "alu_frac": w.relaxations / (rc["layer_loop_ms"] * 1e-3) / 1e9 / ALU_PEAK_GOPS,
+                             "table_bytes": 2 * 4 * w.B * w.S * sbc.shape.m_pitch,
+                             "note": "optimum per instance without a plan; same relaxations, two-layer rolling buffer"}
+        del sbc
+        torch.cuda.empty_cache()
         others = {}
         for k in (0, 1, 2, 4):
             wk = workload_for(k)

@@ -144,9 +144,14 @@ size_t galv_dp_workspace_bytes(const galv_ctx* ctx, const galv_shape* shape);
  * Pad columns M < m < m_pitch are written as GALV_INF / 255.
  * workspace: 256-byte aligned, at least galv_dp_workspace_bytes(shape) bytes,
  * overwritten by every call (calls sharing a workspace must not overlap).
- * With the full table and no argmin table all layers run in ONE cooperative launch (its CTAs hand
+ * Without GALV_STORE_C_FULL two layers roll in the workspace (which then holds
+ * 2*B*S*m_pitch more int32): with GALV_STORE_ARGMIN the plan comes from A, with
+ * neither flag the search yields the optimum only (C_last, and opt_cost from
+ * galv_backtrack with plan = NULL) at a two-layer memory footprint.
+ * Without an argmin table all layers run in ONE cooperative launch (its CTAs hand
  * finished tiles to one another through counters in the workspace, with bounded
- * waits); otherwise, or with GALV_KERNEL_PER_LAYER, one launch per layer.
+ * waits; on the rolling buffer a tile also waits for the readers of the cells it
+ * overwrites); with an argmin table, or with GALV_KERNEL_PER_LAYER, one launch per layer.
  * Nothing synchronises the host, so the call may be captured in a CUDA graph.
  */
 int galv_dp_search(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,

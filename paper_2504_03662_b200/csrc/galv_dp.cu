@@ -421,6 +421,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     __shared__ int desc_count;                             // records posted so far
     __shared__ int drained_count, published_count;         // store warp -> publisher: items whose stores are complete; and back
     __shared__ int store_exit;                             // the store warp has left
+    __shared__ int deps_ok;                                // rolling buffer: items whose dependency wait the producer has passed
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
@@ -451,6 +452,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
         drained_count = 0;
         published_count = 0;
         store_exit = 0;
+        deps_ok = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -518,8 +520,10 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                 // lane 0's TMA loads.  The writes the counters stand for were pushed through the publisher's
                 // proxy fence before its release, so no fence is needed here (it would cost this warp
                 // thousands of cycles per item while the SM's own stores are in flight).
+                // With the two-layer rolling buffer this item overwrites what layer l-2 left there, which the
+                // items of layer l-1 on this tile and the kdep after it still read: it waits for those too.
                 bool ok = true;
-                const int tlast = min(pos.mt, cur.ntp - 1);              // tiles the previous layer did not run store nothing
+                const int tlast = min(pos.mt + (a.C ? 0 : kdep), cur.ntp - 1);   // tiles the previous layer did not run store nothing
                 for (int t0 = max(0, pos.mt - kdep); t0 <= tlast && ok; t0 += 32) {
                     const int t = t0 + lane;
                     if (t <= tlast) {
@@ -539,6 +543,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                     return;
                 }
             }
+            if (MULTI && tile_done && !a.C && lane == 0) st_release_cta(&deps_ok, it + 1);   // the helper may write into the buffer now
             const Item nxt = decode(g_next);              // its instance index lands while this item's stages are awaited
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
@@ -638,6 +643,17 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             }
             if (pos.mt == 0) {
                 // Cells no column maps to: m < mem(l,s), and the pad columns.
+                if (MULTI && tile_done && !a.C) {
+                    // rolling buffer: the cells still hold layer l-2, which layer l-1 may be reading
+                    WaitClock wc;
+                    while (ld_acquire_cta(&deps_ok) <= it) {
+                        if (wc.expired()) {
+                            if (lane == 0) atomicExch(a.err, 1);
+                            return;
+                        }
+                        __nanosleep(100);
+                    }
+                }
                 int32_t* out = a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice;
                 uint8_t* aout = ARG ? a.A + ((size_t)i * a.Lmax + l) * slice : nullptr;
                 for (int c = 0; c < sbw; ++c) {
@@ -1159,8 +1175,8 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     }
     // All layers in one cooperative launch when the grid's CTAs can be co-resident (they wait on one
     // another's tiles); with an argmin table, on request, or for the reference kernel: one launch per layer.
-    // (with the two-layer rolling buffer a layer would overwrite cells a slower CTA still reads)
-    const bool persistent = !reference && a.C && !a.A && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
+    // With the two-layer rolling buffer an item also waits for the readers of the cells it overwrites.
+    const bool persistent = !reference && !a.A && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
     DpArgs ap = a;
     ap.withhold = (sh->flags & GALV_DEBUG_WITHHOLD_LOAD) != 0;
     if (!(sh->flags & GALV_SKIP_INFEASIBLE)) ap.front = nullptr;

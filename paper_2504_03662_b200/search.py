@@ -52,8 +52,8 @@ class SearchBuffers:
         self.workspace = torch.empty(max(256, galv.galv_dp_workspace_bytes(self.shape)), dtype=torch.uint8, device=dev)
         self.status = torch.zeros(B, **i32)
         self.opt_cost = torch.empty(B, **i32)
-        self.plan = torch.empty(B, Lm, **i32)
-        self.mem_used = torch.empty(B, **i32)
+        self.plan = torch.full((B, Lm), -1, **i32)             # stays -1 / 0 when no table is kept (cost-only search)
+        self.mem_used = torch.zeros(B, **i32)
 
     def eval_costs(self, want_fp64: bool = False):
         w = self.w
@@ -72,8 +72,10 @@ class SearchBuffers:
     def backtrack(self, budget: Optional[torch.Tensor] = None, use_A: Optional[bool] = None):
         A = self.A if (use_A is None or use_A) else None
         C = self.C if (use_A is None or not use_A) else None
+        walk = C is not None or A is not None                   # a plan needs one of the tables
         self.galv.galv_backtrack(self.shape, self.L, self.time_q, self.mem_q, self.trans_q, C, A, self.C_last,
-                                 budget, self.opt_cost, self.plan, self.mem_used, self.status)
+                                 budget, self.opt_cost, self.plan if walk else None, self.mem_used if walk else None,
+                                 self.status)
 
     def step(self):
         """One pass of the whole path on the current stream (asynchronous)."""

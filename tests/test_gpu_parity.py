@@ -381,3 +381,46 @@ def test_kernel_span_statistics(galv):
     assert galv.galv_layer_loop_ms_stats()[3] == 64
     galv.galv_set_profiling(False)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("flags", [0, 1024])
+@pytest.mark.parametrize("k", range(len(SHAPES)))
+def test_cost_only_search_on_the_rolling_buffer(orc, galv, flags, k):
+    """No table kept: two layers roll in the workspace (all layers still one launch, an item also waits for
+    the readers of the cells it overwrites); the last layer and the optimum must equal the oracle's."""
+    import torch
+    from paper_2504_03662_b200.search import SearchBuffers
+    B, Lmax, S, M, kw = SHAPES[k]
+    w = inputs.random_tables(700 + k, B, Lmax, S, M, **kw)
+    sb = SearchBuffers(galv, w, flags)
+    assert sb.C is None and sb.A is None
+    for _ in range(2):                                       # the second run starts from used buffers
+        sb.dp_search(); sb.backtrack()
+        res = sb.results()
+        for i in range(B):
+            Li = int(w.L[i])
+            r = orc.search(w.time_q[i, :Li], w.mem_q[i, :Li], w.trans_q[i], M)
+            assert res["status"][i] == r["status"] and res["opt_cost"][i] == r["opt_cost"], i
+            assert (res["plan"][i] == -1).all() and res["mem_used"][i] == 0          # no table, no walk
+            if r["C"] is not None:
+                assert (sb.C_last[i, :, :M + 1].t().cpu().numpy() == r["C"][Li - 1]).all(), i
+
+
+def test_cost_only_search_many_layers_against_full_table(galv):
+    """Rolling buffer under load: many instances, tiles and layers; the last layer must equal the full-table run's."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    for seed, (B, Lmax, S, M, kw) in enumerate([(96, 40, 32, 2048, dict(mem_lo=8, mem_hi=128)),
+                                                (40, 25, 64, 3000, dict(mem_lo=1, mem_hi=900, ragged=True)),
+                                                (300, 12, 24, 700, dict(mem_lo=0, mem_hi=40, ragged=True))]):
+        w = inputs.random_tables(8100 + seed, B, Lmax, S, M, **kw)
+        full = SearchBuffers(galv, w, gb.STORE_C_FULL)
+        full.dp_search(); full.backtrack()
+        lean = SearchBuffers(galv, w, 0)
+        for _ in range(3):
+            lean.dp_search(); lean.backtrack()
+            torch.cuda.synchronize()
+            assert torch.equal(lean.status, full.status) and torch.equal(lean.opt_cost, full.opt_cost)
+            ok = full.status == 0
+            assert torch.equal(lean.C_last[ok], full.C_last[ok])
