@@ -33,20 +33,27 @@ namespace {
 
 constexpr int kInf = GALV_INF;
 constexpr int TS = 8;                 // strategies per warp register tile
-// Every device-side wait gives up after about a second (SM clock cycles; checked every few polls):
-// the role sets the error flag and returns, the host sees GALV_STATUS_TIMEOUT, the context stays usable.
+// Every device-side wait gives up after about a second of waiting (SM clock cycles; checked every 256
+// polls): the role sets the error flag and returns, the host sees GALV_STATUS_TIMEOUT, the context stays
+// usable.  Time is summed poll interval by poll interval with each interval capped, so that a gap in which
+// the whole grid was off the GPU (preemption, time slicing) counts as one interval, not as a timeout.
 constexpr long long kWaitLimitCycles = 2000000000LL;
+constexpr long long kWaitStepCap = 50000000LL;
 
 struct WaitClock {
-    long long t0;
+    long long last, waited;
     int polls;
-    __device__ WaitClock() : t0(0), polls(0) {}
+    __device__ WaitClock() : last(0), waited(0), polls(0) {}
     // true when the limit ran out
     __device__ bool expired() {
         if ((++polls & 255) != 0) return false;
         const long long now = clock64();
-        if (t0 == 0) { t0 = now; return false; }
-        return now - t0 > kWaitLimitCycles;
+        if (last != 0) {
+            const long long step = now - last;
+            waited += step < kWaitStepCap ? step : kWaitStepCap;
+        }
+        last = now;
+        return waited > kWaitLimitCycles;
     }
 };
 
