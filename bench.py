@@ -171,14 +171,18 @@ def time_steps(torch, fn, steps, warmup, barrier):
         fn()
     torch.cuda.synchronize()
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record()
+    for k in range(steps):
         fn()
-    e1.record()
+        ev[k + 1].record()                                       # between steps: lets median and best be reported
     torch.cuda.synchronize()
     barrier()
-    return e0.elapsed_time(e1) * 1e-3
+    LAST_STEP_MS[:] = [ev[k].elapsed_time(ev[k + 1]) for k in range(steps)]
+    return ev[0].elapsed_time(ev[steps]) * 1e-3
+
+
+LAST_STEP_MS: list = []       # per-step durations of the most recent time_steps call
 
 
 def cost_model_scaled(torch, galv, hbm_gbs, barrier, copies=8192):
@@ -217,13 +221,14 @@ def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):
         sb.step()
     galv.galv_set_profiling(True)                                # one event pair around the layer launches of every timed search
     t = time_steps(torch, sb.step, steps, 0, barrier)
+    step_ms = sorted(LAST_STEP_MS)
     layer_ms, layer_min, layer_max, layer_n = galv.galv_layer_loop_ms_stats()   # mean over the timed searches (the last 64)
     galv.galv_set_profiling(False)
     res = sb.results()
     out = {"seconds": t, "ms_per_step": t / steps * 1e3, "cells_per_s": w.cells * steps / t,
            "relax_per_s": w.relaxations * steps / t, "searches_per_s": w.B * steps / t,
            "layer_kernel_ms_avg": layer_ms / max(1, w.Lmax - 1), "layer_loop_ms": layer_ms,
-           "layer_loop_ms_min": layer_min, "layer_loop_ms_max": layer_max, "layer_loop_launches_timed": layer_n,
+           "ms_median": statistics.median(step_ms), "ms_best": step_ms[0], "layer_loop_ms_min": layer_min, "layer_loop_ms_max": layer_max, "layer_loop_launches_timed": layer_n,
            "feasible": int((res["status"] == 0).sum()), "opt_cost_sum": int(res["opt_cost"][res["status"] == 0].sum())}
     return sb, out
 
@@ -304,7 +309,7 @@ def main():
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": t / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": t / args.steps * 1e3, "ms_median": r["ms_median"], "ms_best": r["ms_best"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "Lmax": w.Lmax, "S": w.S, "M": w.M, "per_gpu_batch": w.B,
                    "tables": "full C kept (int32), plan re-derived along the path",
@@ -394,8 +399,10 @@ def main():
         max_layers = max(2, min(w.Lmax, int(2.5e8 * 10.0 / ((w.M + 1) * w.S * w.S)) + 1))   # ~10 s of work per thread
         items, cells = oracle_sample(w, max_layers, threads)
         tc = oracle_run(w, items, threads)
+        t1 = oracle_run(w, items[:1], 1)                          # the same search on one core
         line["cpu_baseline"] = {"value": cells / tc, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": tc,
-                                "sample": f"first {len(items)} instances x first {max_layers} layers, one instance per thread"}
+                                "sample": f"first {len(items)} instances x first {max_layers} layers, one instance per thread",
+                                "single_core_value": cells / len(items) / t1}
     elif rank == 0:
         line["cpu_baseline"] = None
 
