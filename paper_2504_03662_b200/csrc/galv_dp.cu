@@ -1195,10 +1195,20 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     }
     const int pk = ctx->prof_count % 64;
     if (ctx->profiling) cudaEventRecord(ctx->pev[2 * pk], st);
+    bool persistent_ran = false;
     if (persistent) {
-        if ((e = launch_tiled<false>(ap, pl, 1, Lmax, st, maps)) != cudaSuccess) return e;
+        e = launch_tiled<false>(ap, pl, 1, Lmax, st, maps);
+        if (e == cudaErrorCooperativeLaunchTooLarge) {
+            // the grid cannot be co-resident right now (SMs taken by another context): one launch per layer instead
+            (void)cudaGetLastError();
+            ap.tile_done = nullptr;
+        } else if (e != cudaSuccess) {
+            return e;
+        } else {
+            persistent_ran = true;
+        }
     }
-    for (int l = 1; l < Lmax && !persistent; ++l) {
+    for (int l = 1; l < Lmax && !persistent_ran; ++l) {
         if (reference) {
             const int mchunks = (a.m_pitch + 255) / 256;
             layer_reference_kernel<<<dim3((unsigned)((size_t)B * mchunks), S, 1), 256, 0, st>>>(a, l);
