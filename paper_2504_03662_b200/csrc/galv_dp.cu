@@ -551,7 +551,6 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                 }
             }
             if (MULTI && tile_done && !a.C && lane == 0) st_release_cta(&deps_ok, it + 1);   // the helper may write into the buffer now
-            const Item nxt = decode(g_next);              // its instance index lands while this item's stages are awaited
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
             const int yc = row0 + i * inst_rows;
@@ -593,7 +592,9 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                 }
                 __syncwarp();
             }
-            cur = nxt;
+            // Only now the next item: its decoding waits for loads of its own (layer bounds, instance index),
+            // which must not sit between this item's dependency wait and its loads.
+            cur = decode(g_next);
         }
     }
     if (warp == NC + 1) {
