@@ -539,7 +539,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                         const int need = ran[t] * pl.nsb;
                         while (ld_acquire_gpu(c) < need) {
                             if (wc.expired()) { ok = false; break; }
-                            __nanosleep(200);
+                            __nanosleep(100);
                         }
                     }
                     ok = __all_sync(0xffffffffu, ok);
@@ -782,7 +782,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
-                __nanosleep(400);
+                __nanosleep(100);
             }
             if (drained == published) return;                     // the store warp has left and nothing is pending
             if (lane == 0) {
