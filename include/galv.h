@@ -63,6 +63,9 @@ extern "C" {
                                   for galv_dp_search, galv_backtrack, galv_plan_cost, galv_search_host, galv_graph_create */
 #define GALV_KERNEL_REFERENCE 256 /* run the recurrence with the simple one-thread-per-cell kernel (slow; cross-checks) */
 #define GALV_KERNEL_PER_LAYER 512 /* one launch per layer instead of one cooperative launch over all layers */
+#define GALV_KERNEL_NO_PACKED 4096 /* never take the packed 16-bit path (two relaxations per instruction on rebased
+                                      costs; taken on its own when S <= 64, S % 4 == 0, no argmin table, all layers in
+                                      one launch and every transition entry <= 32767; same results) */
 #define GALV_DEBUG_WITHHOLD_LOAD 2048 /* test hook for the time-out path: one CTA never receives its first stage, every
                                          bounded wait that depends on it runs out (about a second each), status gets
                                          GALV_STATUS_TIMEOUT and the call's results are void; nothing faults or hangs */

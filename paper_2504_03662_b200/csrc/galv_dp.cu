@@ -186,7 +186,10 @@ __global__ void validate_kernel(int B, int Lmax, int S, int M, long long tl, con
         else if (s_sum + (long long)(Li - 1) * s_tmax >= (long long)kInf) st = GALV_STATUS_OVERFLOW_RISK;
         status[i] = st;
         // largest shift of a stored row over the valid instances (M+1 stands for "fills the whole row")
-        if (st == 0) atomicMax(maxmem, min(s_mmax, M + 1));
+        if (st == 0) {
+            atomicMax(maxmem, min(s_mmax, M + 1));
+            atomicMax(maxmem + 1, s_tmax);                     // largest transition entry: decides the 16-bit path
+        }
         s_bad = st;
     }
     __syncthreads();
@@ -248,9 +251,12 @@ __device__ long long block_scan_1024(long long v, long long* warp_sums, long lon
 __global__ void __launch_bounds__(1024) schedule_kernel(int B, int Lmax, int M, int tmb, int ntiles_m, int nsb, const int32_t* __restrict__ L,
                                 const int32_t* __restrict__ status, int32_t* __restrict__ order, int32_t* __restrict__ nactive,
                                 int32_t* __restrict__ scratch, const int32_t* __restrict__ minmem_l, int32_t* __restrict__ ntiles,
-                                long long* __restrict__ istart, int32_t* __restrict__ tcount)
+                                long long* __restrict__ istart, int32_t* __restrict__ tcount, int p16_possible,
+                                int32_t* __restrict__ maxmem)
 {
     __shared__ long long warp_sums[32];
+    // The packed 16-bit path needs every trans entry, and twice the largest plus one, to fit 16 bits.
+    if (threadIdx.x == 0) maxmem[2] = (p16_possible && maxmem[1] <= 32767) ? 1 : 0;
     int32_t* hist = scratch;
     int32_t* fill = scratch + Lmax + 2;
     for (int i = threadIdx.x; i < B; i += blockDim.x)
@@ -349,6 +355,22 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
     if (a.A) a.A[(((size_t)i * a.Lmax + l) * a.S + s) * a.m_pitch + m] = (uint8_t)arg;
 }
 
+// ---------------------------------------------------------------- packed trans rows (16-bit path)
+
+// trans_p[i][(l)][q][s] = T[2q][s] | T[2q+1][s] << 16 (the low 16 bits of each; used only when they all fit)
+__global__ void pack_trans_kernel(long long n_mats, int S, const int32_t* __restrict__ trans_q, uint32_t* __restrict__ trans_p)
+{
+    const long long n = n_mats * (S / 2) * S;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+        const int s = (int)(e % S);
+        const long long mq = e / S;
+        const int q = (int)(mq % (S / 2));
+        const long long mat = mq / (S / 2);
+        const int32_t* T = trans_q + mat * S * S;
+        trans_p[e] = ((uint32_t)T[(2 * q) * S + s] & 0xffffu) | ((uint32_t)T[(2 * q + 1) * S + s] << 16);
+    }
+}
+
 // ---------------------------------------------------------------- tiled layer kernel
 //
 // Work items are (layer, instance, m'-tile, s-block), numbered layer by layer.  CTAs take them one
@@ -402,7 +424,17 @@ constexpr int kDescRing = 16;
 // stage a small record the producer fills for the item whose last chunk sits in that stage:
 // mem(l,s) and time(l,s) of the s-block and the instance index; then the staging tile of the
 // outputs and its header.
-template <int TM, int NSG, int NMS, bool ARG, bool MULTI>
+//
+// Packed 16-bit variant (P16): min-plus is invariant under a shift of all candidates of a column, and a
+// candidate more than the largest trans entry above the column's smallest previous-layer value can never
+// win.  So per column m' the previous-layer values are rebased to d = min(c - min_s' c, maxT + 1), which fits
+// 16 bits whenever 2 * maxT + 1 does, and two of them (rows 2q and 2q+1) share a register, as do the two
+// trans entries T[2q][s], T[2q+1][s] (packed once per call).  One __viaddmin_u16x2 then does two relaxations;
+// the result is min(low half, high half) + the column's base.  Exact: only differences are formed, nothing
+// is rounded, clamped candidates stay above every possible winner.  The whole tile (all S rows) comes from
+// the table as int32 into ONE buffer and is rebased by the consumer warps into one of two packed stages, so
+// the next tile's load runs under this tile's inner loop.
+template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false>
 __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
                                                                               const __grid_constant__ CUtensorMap map_t)
@@ -416,6 +448,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     constexpr int RS = TMB + 4;                           // staging row: TMB columns + room for the shift
     constexpr int KU = ARG ? 4 : 16;                      // k-steps per trip of the inner loop
     static_assert(TMB % BOXC == 0 && BOXC % (32 * TM) == 0, "a warp's columns must sit inside one box");
+    static_assert(!(ARG && P16) && (!P16 || MULTI), "the packed path keeps no argmin and runs all layers in one launch");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
@@ -429,10 +462,15 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     __shared__ int drained_count, published_count;         // store warp -> publisher: items whose stores are complete; and back
     __shared__ int store_exit;                             // the store warp has left
     __shared__ int deps_ok;                                // rolling buffer: items whose dependency wait the producer has passed
+    __shared__ __align__(8) uint64_t conv_bar[16];         // packed path: the warps of a column group have rebased their columns
+
+    // Which of the two one-launch kernels runs is decided on the device (largest transition entry).
+    if (MULTI && (a.maxmem[2] != 0) != P16) return;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
-    const int KS = pl.ks, NKC = pl.nkc, NST = pl.nst;
+    const int KS = P16 ? S : pl.ks, NKC = P16 ? 1 : pl.nkc, NST = P16 ? 2 : pl.nst;
+    const int Q = S / 2;                                   // packed path: row pairs
     const int l_last = MULTI ? l_last_arg : l_first + 1;  // single-layer instantiation: loops over l run once
     int32_t* const tile_done = MULTI ? a.tile_done : nullptr;
 
@@ -442,9 +480,13 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     // Items are handed out in increasing order and read only items of the layer before, so the
     // lowest unfinished item can always run: the waits end.
 
-    // stage: NBOX boxes of [KS][BOXC] previous-layer values, then [KS][SB] trans values; 128-byte multiples
-    int32_t* const stage0 = reinterpret_cast<int32_t*>(smem_raw);
-    const int stage_elems = (KS * (TMB + SB) + 31) & ~31;
+    // stage: NBOX boxes of [KS][BOXC] previous-layer values, then [KS][SB] trans values; 128-byte multiples.
+    // Packed path: the raw tile (NBOX boxes of [S][BOXC]) first, then two stages of [Q][TMB] packed values,
+    // [Q][SB] packed trans entries and [TMB] column bases.
+    int32_t* const raw0 = reinterpret_cast<int32_t*>(smem_raw);
+    const int raw_elems = P16 ? ((S * TMB + 31) & ~31) : 0;
+    int32_t* const stage0 = raw0 + raw_elems;
+    const int stage_elems = P16 ? ((Q * TMB + Q * SB + TMB + 31) & ~31) : ((KS * (TMB + SB) + 31) & ~31);
     int32_t* const meta0 = stage0 + NST * stage_elems;
     // staging tile [SB][RS] + its header: mem(l,s) per row, instance, last-layer flag
     int32_t* const stg0 = meta0 + ((NST * META + 31) & ~31);
@@ -453,6 +495,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     if (tid == 0) {
         for (int k = 0; k < NST; ++k) { mbar_init(&full_bar[k], 2); mbar_init(&empty_bar[k], NC); }
         mbar_init(&out_full, NC);
+        for (int k = 0; k < NMS; ++k) mbar_init(&conv_bar[k], NSG);
         out_drained = 0;
         fill_count = 0;
         desc_count = 0;
@@ -465,6 +508,12 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     __syncthreads();
 
     const size_t slice = (size_t)S * m_pitch;
+    // Bounded wait (producer, helper) until the stage of chunk n may be refilled.  Packed path: until every
+    // consumer warp has rebased the item before, which frees the raw buffer and, two items back, the stage.
+    auto stage_free = [&](int n) -> bool {
+        if (P16) return n < 1 || mbar_wait_idle(&empty_bar[0], (n - 1) & 1);
+        return n < NST || mbar_wait_idle(&empty_bar[n % NST], ((n / NST) - 1) & 1);
+    };
 
     if (warp == NC) {
         // ------------------------------------------------------------ producer
@@ -509,7 +558,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             if (last) {
                 // the consumers learn it through a stage that carries no data
                 const int st = n % NST;
-                if (n >= NST && !mbar_wait_idle(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                if (!stage_free(n)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
@@ -558,9 +607,30 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             const int yt = a.trans_layer ? (i * a.Lmax + l) * S : i * S;     // row of trans(0, .) in the tensor map
             // a tile wholly below the previous layer's feasibility frontier reads nothing but +inf: no loads
             const bool skip = a.front && m0 + TMB - 1 < a.front[(size_t)i * a.Lmax + (l - 1)];
-            for (int kc = 0; kc < NKC; ++kc, ++n) {
+            if constexpr (P16) {
+                // one raw tile and one stage of packed trans rows per item; the raw buffer is free once every
+                // consumer warp has rebased the item before (which also means the stage of two items ago is free)
+                const int st = n & 1;
+                if (!stage_free(n)) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+                if (skip) {
+                    if (lane == 0) mbar_arrive(&full_bar[st]);
+                } else if (!((a.withhold & 1) && blockIdx.x == 0 && n == 0) && lane == 0) {
+                    mbar_expect_tx(&full_bar[st], (uint32_t)(S * TMB + Q * SB) * 4u);
+#pragma unroll
+                    for (int bx = 0; bx < NBOX; ++bx)
+                        tma_load_2d(raw0 + bx * S * BOXC, &map_c, m0 + bx * BOXC, yc, &full_bar[st]);
+                    tma_load_2d(stage0 + st * stage_elems + Q * TMB, &map_t, 0,
+                                (a.trans_layer ? i * a.Lmax + l : i) * Q, &full_bar[st]);
+                }
+                __syncwarp();
+                ++n;
+            }
+            for (int kc = 0; kc < (P16 ? 0 : NKC); ++kc, ++n) {
                 const int st = n % NST;
-                if (n >= NST && !mbar_wait_idle(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                if (!stage_free(n)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
@@ -617,7 +687,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             ItemPos pos = {0, d.z, d.w};
             if (l < 0) {
                 const int st = n % NST;
-                if (n >= NST && !mbar_wait_idle(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                if (!stage_free(n)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
@@ -635,7 +705,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             const int tq1 = lane + 32 < sbw ? __ldg(a.time_q + qrow + lane + 32) : 0;
             for (int kc = 0; kc < NKC; ++kc, ++n) {
                 const int st = n % NST;
-                if (n >= NST && !mbar_wait_idle(&empty_bar[st], ((n / NST) - 1) & 1)) {
+                if (!stage_free(n)) {
                     if (lane == 0) atomicExch(a.err, 1);
                     return;
                 }
@@ -813,6 +883,142 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             if (wc.expired()) return false;
         return true;
     };
+    if constexpr (P16) {
+        // ------------------------------------------------------------ consumers, packed 16-bit path
+        constexpr int CW = (32 * TM + NSG - 1) / NSG;      // columns of the group each of its warps rebases
+        constexpr int H = CW <= 16 ? 2 : 1;                // lanes per column (each takes S / H rows)
+        constexpr int LPC = 32 / H;                        // columns a warp handles at a time
+        const int K = a.maxmem[1] + 1;                     // a candidate this far above the column's best cannot win
+        const int rows = S / H;                            // S % 4 == 0: whole row pairs per lane
+        for (int it = 0;; ++it) {
+            const int st = it & 1;
+            if (!mbar_wait(&full_bar[st], (it >> 1) & 1)) {
+                if (lane == 0) atomicExch(a.err, 1);
+                return;
+            }
+            const int4 d = desc[it % kDescRing];
+            if (d.x < 0) {                                  // no more items: wake the store warp (once the previous item is out)
+                if (!drained_wait(it)) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&out_full);
+                return;
+            }
+            const int mw = d.z * TMB + ms * (32 * TM);      // first column of this warp
+            const int nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
+            int32_t* const stg = stage0 + st * stage_elems;
+            uint32_t* const pkc = reinterpret_cast<uint32_t*>(stg);
+            const uint32_t* const pkt = reinterpret_cast<const uint32_t*>(stg + Q * TMB);
+            int32_t* const basep = stg + Q * TMB + Q * SB;
+            const int32_t* const meta = meta0 + st * META;
+            const bool skipped = meta[2 * SB + 1] != 0;     // nothing but +inf to read: no data was loaded
+            if (!skipped) {
+                // rebase: this warp's share of the group's columns, every row of them
+                const int cl = lane % LPC, h = lane / LPC;
+                const int cend = min(sg * CW + CW, 32 * TM);
+                for (int c0 = sg * CW; c0 < cend; c0 += LPC) {
+                    const int cg = c0 + cl;                     // column inside the group
+                    const int c = ms * (32 * TM) + min(cg, 32 * TM - 1);
+                    const int32_t* rp = raw0 + (c / BOXC) * (S * BOXC) + (c % BOXC) + h * rows * BOXC;
+                    int mn = kInf;
+                    for (int r = 0; r < rows; ++r) mn = min(mn, rp[r * BOXC]);
+                    if (H == 2) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, LPC));
+                    if (cg < cend) {
+                        for (int q = 0; q < rows / 2; ++q) {
+                            const int d0 = __viaddmin_s32(rp[(2 * q) * BOXC], -mn, K);
+                            const int d1 = __viaddmin_s32(rp[(2 * q + 1) * BOXC], -mn, K);
+                            pkc[(h * (rows / 2) + q) * TMB + c] = (uint32_t)d0 | ((uint32_t)d1 << 16);
+                        }
+                        if (h == 0) basep[c] = mn;
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&empty_bar[0]);                 // this warp is done with the raw tile
+                mbar_arrive(&conv_bar[ms]);                 // and its columns are there for the group
+            }
+            if (!mbar_wait(&conv_bar[ms], it & 1)) {
+                if (lane == 0) atomicExch(a.err, 1);
+                return;
+            }
+#pragma unroll
+            for (int j = 0; j < TM; ++j)
+#pragma unroll
+                for (int u = 0; u < TS; ++u) acc[j][u] = -1;   // 0xffff in both halves
+            if (!skipped && nj > 0) {
+                const uint32_t* pc = pkc + ms * (32 * TM) + lane;
+                const uint32_t* pt = pkt + sg * TS;
+                int q = 0;
+                auto steps = [&](auto ku) {
+                    constexpr int KQ = decltype(ku)::value;
+                    for (; q + KQ <= Q; q += KQ) {
+#pragma unroll
+                        for (int kk = 0; kk < KQ; ++kk) {
+                            uint32_t c[TM];
+#pragma unroll
+                            for (int j = 0; j < TM; ++j) c[j] = pc[kk * TMB + j * 32];
+                            const uint4 t0 = *reinterpret_cast<const uint4*>(pt + kk * SB);
+                            const uint4 t1 = *reinterpret_cast<const uint4*>(pt + kk * SB + 4);
+                            const uint32_t t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                            for (int j = 0; j < TM; ++j)
+#pragma unroll
+                                for (int u = 0; u < TS; ++u)
+                                    acc[j][u] = (int)__viaddmin_u16x2(c[j], t[u], (uint32_t)acc[j][u]);
+                        }
+                        pc += KQ * TMB;
+                        pt += KQ * SB;
+                    }
+                };
+                steps(std::integral_constant<int, 16>());
+                steps(std::integral_constant<int, 4>());
+                steps(std::integral_constant<int, 1>());
+            }
+            int mm[TS], tt[TS];
+            {
+                const int4 m0v = *reinterpret_cast<const int4*>(meta + sg * TS);
+                const int4 m1v = *reinterpret_cast<const int4*>(meta + sg * TS + 4);
+                const int4 t0v = *reinterpret_cast<const int4*>(meta + SB + sg * TS);
+                const int4 t1v = *reinterpret_cast<const int4*>(meta + SB + sg * TS + 4);
+                mm[0] = m0v.x; mm[1] = m0v.y; mm[2] = m0v.z; mm[3] = m0v.w; mm[4] = m1v.x; mm[5] = m1v.y; mm[6] = m1v.z; mm[7] = m1v.w;
+                tt[0] = t0v.x; tt[1] = t0v.y; tt[2] = t0v.z; tt[3] = t0v.w; tt[4] = t1v.x; tt[5] = t1v.y; tt[6] = t1v.z; tt[7] = t1v.w;
+            }
+            int bs[TM];
+#pragma unroll
+            for (int j = 0; j < TM; ++j) bs[j] = (skipped || j >= nj) ? kInf : basep[ms * (32 * TM) + j * 32 + lane];
+            if (!drained_wait(it)) {                         // the previous item has been drained
+                if (lane == 0) atomicExch(a.err, 1);
+                return;
+            }
+            {
+                const int s0l = sg * TS;
+                const int col = ms * (32 * TM) + lane;
+#pragma unroll
+                for (int u = 0; u < TS; ++u) {
+                    int32_t* R = stg0 + (s0l + u) * RS + (mm[u] & 3) + col;
+#pragma unroll
+                    for (int j = 0; j < TM; ++j)
+                        if (j < nj) {
+                            const uint32_t x = (uint32_t)acc[j][u];
+                            const int w = (int)min(x & 0xffffu, x >> 16);         // the better of the two row parities
+                            const int v = __viaddmin_s32(bs[j], w, kInf);          // back on the column's base (+inf stays)
+                            R[j * 32] = __viaddmin_s32(v, tt[u], kInf);
+                        }
+                }
+                if (ms == 0) {
+                    int v = mm[0];
+#pragma unroll
+                    for (int u = 1; u < TS; ++u) v = lane == u ? mm[u] : v;
+                    if (lane < TS) hdr0[s0l + lane] = v;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&out_full);            // release: the staging writes come before it
+        }
+    }
     for (int it = 0;; ++it) {
         int l = 0, mw = 0, nj = 0;
         ItemPos pos = {0, 0, 0};
@@ -994,14 +1200,22 @@ __global__ void finalize_kernel(int B, const int32_t* err, int32_t* status)
 // more than one layer means the CTAs wait on one another's tiles, so the launch is cooperative
 // (all CTAs guaranteed co-resident).
 template <int TM, int NSG, int NMS, bool ARG>
-cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_last, cudaStream_t st, const CUtensorMap* maps)
+cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_last, cudaStream_t st, const CUtensorMap* maps,
+                       bool packed)
 {
     auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG, false>;
     auto kern_multi = layer_tiled_kernel<TM, NSG, NMS, false, true>;
+    auto kern_packed = layer_tiled_kernel<TM, NSG, NMS, false, true, true>;
     if (!maps) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_multi, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+        if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         return e;
+    }
+    if (packed) {
+        // the packed 16-bit kernel over all layers: its own tensor maps (whole-tile boxes, packed trans rows)
+        void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[2], (void*)&maps[3]};
+        return cudaLaunchCooperativeKernel((const void*)kern_packed, dim3(pl.grid), dim3((NSG * NMS + 4) * 32), args, (size_t)pl.p16_smem, st);
     }
     if (l_last - l_first > 1) {
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[0], (void*)&maps[1]};
@@ -1013,17 +1227,18 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
 
 // nsg warps along s, 16/nsg (rounded down) along m: one instantiation per s-block width.
 template <bool ARG>
-cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l_first, int l_last, cudaStream_t st, const CUtensorMap* maps)
+cudaError_t launch_tiled(const DpArgs& a, const DpPlan& pl, int l_first, int l_last, cudaStream_t st, const CUtensorMap* maps,
+                         bool packed = false)
 {
     switch (pl.nsg) {
-    case 1: return launch_one<4, 1, 16, ARG>(a, pl, l_first, l_last, st, maps);
-    case 2: return launch_one<4, 2, 8, ARG>(a, pl, l_first, l_last, st, maps);
-    case 3: return launch_one<4, 3, 5, ARG>(a, pl, l_first, l_last, st, maps);
-    case 4: return launch_one<4, 4, 4, ARG>(a, pl, l_first, l_last, st, maps);
-    case 5: return launch_one<4, 5, 3, ARG>(a, pl, l_first, l_last, st, maps);
-    case 6: return launch_one<4, 6, 2, ARG>(a, pl, l_first, l_last, st, maps);
-    case 7: return launch_one<4, 7, 2, ARG>(a, pl, l_first, l_last, st, maps);
-    case 8: return launch_one<4, 8, 2, ARG>(a, pl, l_first, l_last, st, maps);
+    case 1: return launch_one<4, 1, 16, ARG>(a, pl, l_first, l_last, st, maps, packed);
+    case 2: return launch_one<4, 2, 8, ARG>(a, pl, l_first, l_last, st, maps, packed);
+    case 3: return launch_one<4, 3, 5, ARG>(a, pl, l_first, l_last, st, maps, packed);
+    case 4: return launch_one<4, 4, 4, ARG>(a, pl, l_first, l_last, st, maps, packed);
+    case 5: return launch_one<4, 5, 3, ARG>(a, pl, l_first, l_last, st, maps, packed);
+    case 6: return launch_one<4, 6, 2, ARG>(a, pl, l_first, l_last, st, maps, packed);
+    case 7: return launch_one<4, 7, 2, ARG>(a, pl, l_first, l_last, st, maps, packed);
+    case 8: return launch_one<4, 8, 2, ARG>(a, pl, l_first, l_last, st, maps, packed);
     default: return cudaErrorInvalidConfiguration;
     }
 }
@@ -1045,13 +1260,16 @@ WsLayout galv_ws_layout(const galv_shape* sh)
     w.order = off;   off = align256(off + (size_t)sh->B * 4);
     w.nactive = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.scratch = off; off = align256(off + (size_t)4 * (sh->Lmax + 2) * 4);    // two int32 arrays, one 64-bit array
-    w.err = off;     off = align256(off + 8);                  // error flag, largest mem
+    w.err = off;     off = align256(off + 16);                 // error flag, largest mem, largest trans, path chosen
     w.minmem_l = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.ntiles = off;   off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.istart = off;   off = align256(off + (size_t)(sh->Lmax + 1) * 8);
     w.tcount = off;   off = align256(off + (size_t)sh->Lmax * ((sh->M + 128) / 128) * 4);
     w.front = off;    off = align256(off + (size_t)sh->B * sh->Lmax * 4);
     w.tile_done = off; off = align256(off + (size_t)sh->B * ((sh->M + 128) / 128) * 4);   // per (instance, tile of >= 128 columns)
+    w.trans_p = off;                                           // packed trans rows for the 16-bit path (S <= 64, S % 4 == 0)
+    if (sh->S <= 64 && sh->S % 4 == 0)
+        off = align256(off + (size_t)sh->B * ((sh->flags & GALV_TRANS_PER_LAYER) ? sh->Lmax : 1) * (sh->S / 2) * sh->S * 4);
     w.roll = off;
     if (!(sh->flags & GALV_STORE_C_FULL)) off = align256(off + (size_t)2 * sh->B * sh->S * sh->m_pitch * 4);
     w.total = off;
@@ -1094,6 +1312,16 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     pl->ntiles_m = (sh->M + 1 + pl->tmb - 1) / pl->tmb;
     pl->smem = nst * stage_bytes + extra;
     pl->tma_t = (S % 4) == 0;                             // trans row pitch a multiple of 16 bytes
+    // Packed 16-bit path: the whole previous-layer tile (all S rows, one buffer) as it comes from the table, two
+    // stages of its packed form (row pairs), the packed trans rows and the column bases; no argmin table.
+    {
+        const int q = S / 2;
+        const int raw = (S * pl->tmb * 4 + 127) & ~127;
+        const int pst = ((q * pl->tmb + q * pl->sb + pl->tmb) * 4 + 127) & ~127;
+        const int total = raw + 2 * pst + ((2 * (2 * pl->sb + 4) + 31) & ~31) * 4 + staging;
+        pl->p16 = S <= 64 && S % 4 == 0 && pl->nsb == 1 && !(sh->flags & GALV_STORE_ARGMIN) && total <= budget;
+        pl->p16_smem = total;
+    }
     const long long items = (long long)sh->B * pl->ntiles_m * pl->nsb;
     pl->grid = (int)(items < ctx->num_sms ? items : ctx->num_sms);
     return true;
@@ -1141,7 +1369,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     const int B = a.B, Lmax = a.Lmax, S = a.S;
     e = cudaMemsetAsync(a.scratch, 0, (size_t)4 * (Lmax + 2) * 4, st);      // histogram, fill and work counters
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(a.err, 0, 8, st);
+    e = cudaMemsetAsync(a.err, 0, 16, st);
     if (e != cudaSuccess) return e;
     const bool reference = (sh->flags & GALV_KERNEL_REFERENCE) != 0;
     DpPlan pl;
@@ -1150,10 +1378,17 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     if (reference) { pl.tmb = 256; pl.ntiles_m = (a.M + 256) / 256; }
     e = cudaMemsetAsync(a.minmem_l, 0x7f, (size_t)(Lmax + 1) * 4, st);
     if (e != cudaSuccess) return e;
+    // All layers in one cooperative launch when the grid's CTAs can be co-resident (they wait on one
+    // another's tiles); with an argmin table, on request, or for the reference kernel: one launch per layer.
+    // With the two-layer rolling buffer an item also waits for the readers of the cells it overwrites.
+    const bool persistent = !reference && !a.A && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
+    // The packed 16-bit kernel is launched as well when the shape allows it; which of the two runs is decided on
+    // the device, where the largest transition entry is known (the other one returns at once).
+    const int will_p16 = persistent && pl.p16 && !(sh->flags & GALV_KERNEL_NO_PACKED);
     validate_kernel<<<B, 128, 0, st>>>(B, Lmax, S, a.M, (long long)a.trans_layer, a.L, a.time_q, a.mem_q, a.trans_q, a.status, a.err + 1, a.minmem_l,
                                        (sh->flags & GALV_SKIP_INFEASIBLE) ? a.front : nullptr);
     schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.M, pl.tmb, pl.ntiles_m, pl.nsb, a.L, a.status, a.order, a.nactive, a.scratch,
-                                         a.minmem_l, a.ntiles, a.istart, a.tcount);
+                                         a.minmem_l, a.ntiles, a.istart, a.tcount, will_p16, a.err + 1);
     {
         int gx = (a.m_pitch + 255) / 256;
         if (gx > 8) gx = 8;
@@ -1171,7 +1406,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-    CUtensorMap maps[2];
+    CUtensorMap maps[4];
     std::memset(maps, 0, sizeof(maps));
     if (!reference) {
         // previous-layer values as a 2-D tensor [rows of m_pitch columns]; box = ks rows x (<=256) columns
@@ -1180,11 +1415,16 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
         if ((e = encode_2d(&maps[0], a.C ? (void*)a.C : (void*)a.roll, (size_t)a.m_pitch, rows, boxc, pl.ks)) != cudaSuccess) return e;
         if (pl.tma_t &&
             (e = encode_2d(&maps[1], (void*)a.trans_q, (size_t)S, (size_t)B * (a.trans_layer ? Lmax : 1) * S, pl.sb, pl.ks)) != cudaSuccess) return e;
+        if (will_p16) {
+            // whole tiles (all S rows) of the previous layer; packed trans rows [S/2 row pairs][S]
+            const long long n_mats = (long long)B * (a.trans_layer ? Lmax : 1);
+            if ((e = encode_2d(&maps[2], a.C ? (void*)a.C : (void*)a.roll, (size_t)a.m_pitch, rows, boxc, S)) != cudaSuccess) return e;
+            if ((e = encode_2d(&maps[3], (void*)a.trans_p, (size_t)S, (size_t)n_mats * (S / 2), pl.sb, S / 2)) != cudaSuccess) return e;
+            long long blocks = (n_mats * (S / 2) * S + 255) / 256;
+            if (blocks > 148 * 8) blocks = 148 * 8;
+            pack_trans_kernel<<<(int)blocks, 256, 0, st>>>(n_mats, S, a.trans_q, a.trans_p);
+        }
     }
-    // All layers in one cooperative launch when the grid's CTAs can be co-resident (they wait on one
-    // another's tiles); with an argmin table, on request, or for the reference kernel: one launch per layer.
-    // With the two-layer rolling buffer an item also waits for the readers of the cells it overwrites.
-    const bool persistent = !reference && !a.A && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
     DpArgs ap = a;
     ap.withhold = (sh->flags & GALV_DEBUG_WITHHOLD_LOAD) != 0;
     if (!(sh->flags & GALV_SKIP_INFEASIBLE)) ap.front = nullptr;
@@ -1198,7 +1438,9 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     if (ctx->profiling) cudaEventRecord(ctx->pev[2 * pk], st);
     bool persistent_ran = false;
     if (persistent) {
-        e = launch_tiled<false>(ap, pl, 1, Lmax, st, maps);
+        // packed kernel first where possible, then the 32-bit one: each returns at once unless it is the one chosen
+        e = will_p16 ? launch_tiled<false>(ap, pl, 1, Lmax, st, maps, true) : cudaSuccess;
+        if (e == cudaSuccess) e = launch_tiled<false>(ap, pl, 1, Lmax, st, maps);
         if (e == cudaErrorCooperativeLaunchTooLarge) {
             // the grid cannot be co-resident right now (SMs taken by another context): one launch per layer instead
             (void)cudaGetLastError();

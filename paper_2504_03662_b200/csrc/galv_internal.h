@@ -33,6 +33,8 @@ struct DpPlan {
     int threads;   // (nsg * nms + 4) * 32: consumer warps, producer, helper, store and publisher warps
     int smem;      // dynamic shared memory bytes
     int grid;      // resident CTAs
+    int p16;       // the packed 16-bit path is possible for this shape (whether the costs allow it is known on the device)
+    int p16_smem;  // its dynamic shared memory bytes
 };
 
 struct DpArgs {
@@ -54,7 +56,8 @@ struct DpArgs {
     long long* istart;   // [Lmax+1] items of the layers before l (layer 1 starts at 0); [Lmax] = all items
     int32_t* err;        // device error flag
     int32_t* tile_done;  // [B][ntiles_m] finished items per (instance, tile); NULL when layers are separate launches
-    int32_t* maxmem;     // largest mem over the valid instances (min(.., M+1))
+    int32_t* maxmem;     // largest mem over the valid instances (min(.., M+1)); [1] largest trans entry; [2] 1: packed 16-bit path
+    uint32_t* trans_p;   // packed pairs of trans rows for the 16-bit path: [B][(Lmax)][S/2][S], entry = T[2q][s] | T[2q+1][s] << 16
     int32_t* minmem_l;   // [Lmax+1] smallest mem of each layer over the valid instances
     int32_t* front;      // [B][Lmax] feasibility frontier (sum of the layers' smallest mem), or NULL when tiles are never skipped
     int32_t* ntiles;     // [Lmax+1] tiles per instance that can store anything in layer l
@@ -67,7 +70,7 @@ struct DpArgs {
 int galv_set_error(galv_ctx* ctx, int code, const char* text);
 
 // workspace carve-up (offsets in bytes, all 256-aligned)
-struct WsLayout { size_t order, nactive, scratch, err, minmem_l, ntiles, istart, tcount, front, tile_done, roll, total; };
+struct WsLayout { size_t order, nactive, scratch, err, minmem_l, ntiles, istart, tcount, front, tile_done, trans_p, roll, total; };
 WsLayout galv_ws_layout(const galv_shape* sh);
 
 bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* plan);
