@@ -223,11 +223,12 @@ def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):
     t = time_steps(torch, sb.step, steps, 0, barrier)
     step_ms = sorted(LAST_STEP_MS)
     layer_ms, layer_min, layer_max, layer_n = galv.galv_layer_loop_ms_stats()   # mean over the timed searches (the last 64)
+    packed = galv.galv_dp_search_path(sb.shape, sb.workspace)                   # which inner loop ran
     galv.galv_set_profiling(False)
     res = sb.results()
     out = {"seconds": t, "ms_per_step": t / steps * 1e3, "cells_per_s": w.cells * steps / t,
            "relax_per_s": w.relaxations * steps / t, "searches_per_s": w.B * steps / t,
-           "layer_kernel_ms_avg": layer_ms / max(1, w.Lmax - 1), "layer_loop_ms": layer_ms,
+           "layer_kernel_ms_avg": layer_ms / max(1, w.Lmax - 1), "layer_loop_ms": layer_ms, "packed": packed,
            "ms_median": statistics.median(step_ms), "ms_best": step_ms[0], "layer_loop_ms_min": layer_min, "layer_loop_ms_max": layer_max, "layer_loop_launches_timed": layer_n,
            "feasible": int((res["status"] == 0).sum()), "opt_cost_sum": int(res["opt_cost"][res["status"] == 0].sum())}
     return sb, out
@@ -316,8 +317,11 @@ def main():
                    "l2": "tables far larger than L2 (no flush needed)", "parallelism": f"instances x{world}"},
         "searches_per_s": world * w.B * args.steps / t, "relaxations_per_s": world * w.relaxations * args.steps / t,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(w) * args.steps,
-        "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_GOPS, "unit": "G add-min/s",
-                     "frac": achieved / ALU_PEAK_GOPS,
+        "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_GOPS * (2 if r["packed"] else 1), "unit": "G add-min/s",
+                     "frac": achieved / (ALU_PEAK_GOPS * (2 if r["packed"] else 1)),
+                     "frac_of_32bit_peak": achieved / ALU_PEAK_GOPS,
+                     "inner_loop": ("packed 16-bit add-min on rebased costs, two relaxations per instruction" if r["packed"]
+                                    else "32-bit fused add-min, one relaxation per instruction"),
                      "traffic": (NCU_TRAFFIC_BYTES_PER_LAYER[w.name] * (w.Lmax - 1)
                                  if w.name in NCU_TRAFFIC_BYTES_PER_LAYER else None),
                      "traffic_unit": "bytes per launch (ncu dram read+write per layer x layers)",
@@ -326,7 +330,8 @@ def main():
                      "kernel": "layer_tiled_kernel (one cooperative launch over all layers)",
                      "launch_ms": r["layer_loop_ms"], "launch_ms_min": r["layer_loop_ms_min"],
                      "launch_ms_max": r["layer_loop_ms_max"], "launches_timed": r["layer_loop_launches_timed"],
-                     "peak_source": "derived: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min per lane per clock"},
+                     "peak_source": "derived: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min per lane per clock"
+                                    + (" (two relaxations each in the packed 16-bit form)" if r["packed"] else "")},
     }
 
     if rank == 0:
@@ -345,7 +350,7 @@ def main():
         except OSError:
             pass
         hbm_gbs = peaks.get("hbm_gbs", 6650.0)
-        line["roofline"]["t_alu_ms"] = w.relaxations / (ALU_PEAK_GOPS * 1e9) * 1e3
+        line["roofline"]["t_alu_ms"] = w.relaxations / (line["roofline"]["peak"] * 1e9) * 1e3
         line["roofline"]["t_hbm_ms"] = hbm_bytes / (hbm_gbs * 1e9) * 1e3
         line["roofline"]["hbm_peak"] = f"{hbm_gbs} GB/s " + ("of measured" if peaks else "of fallback")
         line["roofline"]["step_frac_of_bound"] = max(line["roofline"]["t_alu_ms"], line["roofline"]["t_hbm_ms"]) / (t / args.steps * 1e3)
@@ -365,7 +370,8 @@ def main():
         sbc, rc = bench_workload(torch, galv, w, max(5, args.steps // 2), 3, barrier, flags=0)
         line["cost_only"] = {"ms_per_step": rc["ms_per_step"], "cells_per_s": rc["cells_per_s"],
                              "searches_per_s": rc["searches_per_s"], "opt_cost_sum": rc["opt_cost_sum"],
-                             "alu_frac": w.relaxations / (rc["layer_loop_ms"] * 1e-3) / 1e9 / ALU_PEAK_GOPS,
+                             "alu_frac": w.relaxations / (rc["layer_loop_ms"] * 1e-3) / 1e9 / (ALU_PEAK_GOPS * (2 if rc["packed"] else 1)),
+                             "packed": rc["packed"],
                              "table_bytes": 2 * 4 * w.B * w.S * sbc.shape.m_pitch,
                              "note": "optimum per instance without a plan; same relaxations, two-layer rolling buffer"}
         del sbc
@@ -375,7 +381,8 @@ def main():
             wk = workload_for(k)
             sbk, rk = bench_workload(torch, galv, wk, max(5, args.steps // 2), 3, barrier)
             o = {key: rk[key] for key in ("ms_per_step", "cells_per_s", "relax_per_s", "searches_per_s")}
-            o["alu_frac"] = rk["relax_per_s"] / (ALU_PEAK_GOPS * 1e9)
+            o["alu_frac"] = rk["relax_per_s"] / (ALU_PEAK_GOPS * 1e9 * (2 if rk["packed"] else 1))
+            o["packed"] = rk["packed"]
             # the same step replayed from a CUDA graph (launch latency matters for the small workloads)
             g = torch.cuda.CUDAGraph()
             s = torch.cuda.Stream()

@@ -164,6 +164,13 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
                    int32_t* status, void* stream);
 
 /*
+ * Which inner loop the most recent galv_dp_search on `workspace` ran: *packed = 1 for the packed
+ * 16-bit one (two relaxations per instruction; see GALV_KERNEL_NO_PACKED), 0 for the 32-bit one.
+ * The choice is made on the device; this call waits for `stream` and reads it back (host pointer).
+ */
+int galv_dp_search_path(galv_ctx* ctx, const galv_shape* shape, const void* workspace, int32_t* packed, void* stream);
+
+/*
  * The same search without any caller-provided scratch (the paper has no
  * counterpart; this exists for deployment).  Some callers cannot call
  * cudaMalloc at all: a plugin running inside a host application that owns the

@@ -25,7 +25,7 @@ STATIC_WORKSPACE_BYTES = 1 << 20
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgalv.so")
 
 EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "galv_eval_costs",
-           "galv_dp_workspace_bytes", "galv_dp_search", "galv_backtrack", "galv_search_host_arena_bytes",
+           "galv_dp_workspace_bytes", "galv_dp_search", "galv_dp_search_path", "galv_backtrack", "galv_search_host_arena_bytes",
            "galv_search_host", "galv_probe_int_alu", "galv_set_profiling", "galv_last_layer_loop_ms", "galv_layer_loop_ms_stats",
            "galv_dp_search_static", "galv_select_best", "galv_prune_strategies",
            "galv_compact_tables", "galv_expand_plan", "galv_plan_cost", "galv_graph_create", "galv_graph_launch",
@@ -67,6 +67,7 @@ def load_library() -> C.CDLL:
     lib.galv_dp_workspace_bytes.argtypes = [vp, shp]
     lib.galv_dp_workspace_bytes.restype = sz
     lib.galv_dp_search.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.galv_dp_search_path.argtypes = [vp, shp, vp, C.POINTER(C.c_int32), vp]
     lib.galv_backtrack.argtypes = [vp, shp] + [vp] * 13
     lib.galv_dp_search_static.argtypes = [vp, shp] + [vp] * 9
     lib.galv_select_best.argtypes = [vp, C.c_int32, C.c_int32] + [vp] * 8
@@ -204,6 +205,12 @@ class Galv:
 
     def galv_stage_partition(self, Lm, P, range_opt, cuts, bottleneck):
         self._check(self.lib.galv_stage_partition(self.h, Lm, P, _ptr(range_opt), _ptr(cuts), _ptr(bottleneck), _stream()))
+
+    def galv_dp_search_path(self, shape, workspace) -> bool:
+        """True when the most recent search on this workspace ran the packed 16-bit inner loop."""
+        out = C.c_int32()
+        self._check(self.lib.galv_dp_search_path(self.h, C.byref(shape), _ptr(workspace), C.byref(out), _stream()))
+        return bool(out.value)
 
     def galv_backtrack(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, budget, opt_cost, plan, mem_used, status):
         self._check(self.lib.galv_backtrack(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),

@@ -208,6 +208,19 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const 
     return e == cudaSuccess ? GALV_OK : cuda_fail(ctx, "galv_dp_search", e);
 }
 
+int galv_dp_search_path(galv_ctx* ctx, const galv_shape* sh, const void* workspace, int32_t* packed, void* stream)
+{
+    if (!ctx) return GALV_ERR_INVALID_ARG;
+    if (!shape_ok(sh) || !workspace || !packed) { set_err(ctx, "galv_dp_search_path: bad shape or NULL pointer"); return GALV_ERR_INVALID_ARG; }
+    const WsLayout w = galv_ws_layout(sh);
+    int32_t flags[4] = {0, 0, 0, 0};                       // error flag, largest mem, largest trans, path
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpy(flags, static_cast<const char*>(workspace) + w.err, sizeof(flags), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(ctx, "galv_dp_search_path", e);
+    *packed = flags[3] != 0;
+    return GALV_OK;
+}
+
 int galv_backtrack(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const int32_t* time_q,
                    const int32_t* mem_q, const int32_t* trans_q, const int32_t* C, const uint8_t* A,
                    const int32_t* C_last, const int32_t* budget, int32_t* opt_cost, int32_t* plan,

@@ -449,3 +449,39 @@ def test_full_parity_every_instance(orc, galv, k):
             assert (res["plan"][i, :Li] == r["plan"]).all() and res["mem_used"][i] == r["mem_used"], i
             assert (sb.table(i)[:Li] == r["C"]).all(), i
         del ref
+
+
+@pytest.mark.parametrize("S,M,B,Lmax", [(64, 1500, 5, 9), (48, 900, 4, 12), (8, 5000, 3, 6), (24, 2881, 6, 7), (4, 300, 2, 5)])
+def test_packed_16bit_path_choice_and_parity(orc, galv, S, M, B, Lmax):
+    """The packed 16-bit inner loop is taken exactly when every transition entry is <= 32767 (and the shape allows
+    it); its tables equal the 32-bit loop's and the oracle's, at the limit and with costs far above 16 bits."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    for top, want in ((32767, True), (32768, False), (5, True)):
+        w = inputs.random_tables(4000 + S + top % 7, B, Lmax, S, M, ragged=True, mem_lo=0, mem_hi=M // 4,
+                                 time_hi=3_000_000, trans_hi=top)
+        w.trans_q[0, 0, min(1, S - 1)] = top                     # the largest entry is really there
+        w.time_q[B - 1, 1, :] = 7                                # a cheap layer: big spreads between strategies elsewhere
+        w.mem_q[0, 2, : S // 2] = M + 5                          # +inf rows in some columns
+        sb = SearchBuffers(galv, w, gb.STORE_C_FULL)
+        sb.dp_search(); sb.backtrack()
+        assert galv.galv_dp_search_path(sb.shape, sb.workspace) == want
+        res = sb.results()
+        plain = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_NO_PACKED)
+        plain.dp_search(); plain.backtrack()
+        assert not galv.galv_dp_search_path(plain.shape, plain.workspace)
+        assert torch.equal(sb.status, plain.status) and torch.equal(sb.opt_cost, plain.opt_cost)
+        for i in range(B):
+            Li = int(w.L[i])
+            assert torch.equal(sb.C[i, :Li], plain.C[i, :Li]), (top, i)
+            r = orc.search(w.time_q[i, :Li], w.mem_q[i, :Li], w.trans_q[i], M)
+            assert res["status"][i] == r["status"] and res["opt_cost"][i] == r["opt_cost"]
+            if r["C"] is not None:
+                assert (sb.table(i)[:Li] == r["C"]).all(), (top, i)
+    # shapes the packed path does not take: S not a multiple of 4, S > 64, an argmin table
+    for S2, flags in ((6, gb.STORE_C_FULL), (70, gb.STORE_C_FULL), (S, gb.STORE_C_FULL | gb.STORE_ARGMIN)):
+        w = inputs.random_tables(77, 2, 4, S2, 200, trans_hi=100)
+        sb = SearchBuffers(galv, w, flags)
+        sb.dp_search()
+        assert not galv.galv_dp_search_path(sb.shape, sb.workspace)
