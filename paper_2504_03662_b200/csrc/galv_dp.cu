@@ -886,10 +886,10 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     if constexpr (P16) {
         // ------------------------------------------------------------ consumers, packed 16-bit path
         constexpr int CW = (32 * TM + NSG - 1) / NSG;      // columns of the group each of its warps rebases
-        constexpr int H = CW <= 16 ? 2 : 1;                // lanes per column (each takes S / H rows)
-        constexpr int LPC = 32 / H;                        // columns a warp handles at a time
+        constexpr int LPC = 16;                            // columns a warp handles at a time: two lanes per column,
+                                                           // each with half of the rows (S / 2 <= 32 values, in registers)
         const int K = a.maxmem[1] + 1;                     // a candidate this far above the column's best cannot win
-        const int rows = S / H;                            // S % 4 == 0: whole row pairs per lane
+        const int rows = S / 2;                            // S % 4 == 0: whole row pairs per lane
         for (int it = 0;; ++it) {
             const int st = it & 1;
             if (!mbar_wait(&full_bar[st], (it >> 1) & 1)) {
@@ -915,22 +915,30 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             const int32_t* const meta = meta0 + st * META;
             const bool skipped = meta[2 * SB + 1] != 0;     // nothing but +inf to read: no data was loaded
             if (!skipped) {
-                // rebase: this warp's share of the group's columns, every row of them
+                // rebase: this warp's share of the group's columns, every row of them, read once
                 const int cl = lane % LPC, h = lane / LPC;
                 const int cend = min(sg * CW + CW, 32 * TM);
                 for (int c0 = sg * CW; c0 < cend; c0 += LPC) {
                     const int cg = c0 + cl;                     // column inside the group
                     const int c = ms * (32 * TM) + min(cg, 32 * TM - 1);
                     const int32_t* rp = raw0 + (c / BOXC) * (S * BOXC) + (c % BOXC) + h * rows * BOXC;
+                    int v[32];
                     int mn = kInf;
-                    for (int r = 0; r < rows; ++r) mn = min(mn, rp[r * BOXC]);
-                    if (H == 2) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, LPC));
+#pragma unroll
+                    for (int r = 0; r < 32; ++r) {
+                        v[r] = r < rows ? rp[r * BOXC] : kInf;
+                        mn = min(mn, v[r]);
+                    }
+                    mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, LPC));
                     if (cg < cend) {
-                        for (int q = 0; q < rows / 2; ++q) {
-                            const int d0 = __viaddmin_s32(rp[(2 * q) * BOXC], -mn, K);
-                            const int d1 = __viaddmin_s32(rp[(2 * q + 1) * BOXC], -mn, K);
-                            pkc[(h * (rows / 2) + q) * TMB + c] = (uint32_t)d0 | ((uint32_t)d1 << 16);
-                        }
+                        uint32_t* out = pkc + (h * (rows / 2)) * TMB + c;
+#pragma unroll
+                        for (int q = 0; q < 16; ++q)
+                            if (2 * q < rows) {
+                                const int d0 = __viaddmin_s32(v[2 * q], -mn, K);
+                                const int d1 = __viaddmin_s32(v[2 * q + 1], -mn, K);
+                                out[q * TMB] = (uint32_t)d0 | ((uint32_t)d1 << 16);
+                            }
                         if (h == 0) basep[c] = mn;
                     }
                 }
