@@ -90,6 +90,9 @@ __device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
 __device__ __forceinline__ void red_relaxed_gpu_add(int32_t* p, int v) {
     asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ void red_release_cta_add(int* p, int v) {
+    asm volatile("red.release.cta.shared::cta.add.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
 __device__ __forceinline__ void st_release_cta(int* p, int v) {
     asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
@@ -435,7 +438,7 @@ constexpr int kDescRing = 16;
 // the table as int32 into ONE buffer and is rebased by the consumer warps into one of two packed stages, so
 // the next tile's load runs under this tile's inner loop.
 template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false>
-__global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
+__global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
                                                                               const __grid_constant__ CUtensorMap map_t)
 {
@@ -447,6 +450,8 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     constexpr int META = 2 * SB + 4;
     constexpr int RS = TMB + 4;                           // staging row: TMB columns + room for the shift
     constexpr int KU = ARG ? 4 : 16;                      // k-steps per trip of the inner loop
+    constexpr int NSW = P16 ? 2 : 1;                      // store warps: the packed path's items are short enough for one
+                                                          // warp's row-by-row issue (about 10k cycles a tile) to hold them up
     static_assert(TMB % BOXC == 0 && BOXC % (32 * TM) == 0, "a warp's columns must sit inside one box");
     static_assert(!(ARG && P16) && (!P16 || MULTI), "the packed path keeps no argmin and runs all layers in one launch");
 
@@ -463,6 +468,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     __shared__ int store_exit;                             // the store warp has left
     __shared__ int deps_ok;                                // rolling buffer: items whose dependency wait the producer has passed
     __shared__ __align__(8) uint64_t conv_bar[16];         // packed path: the warps of a column group have rebased their columns
+    __shared__ int drained_b;                              // second store warp -> first: items whose rows it has stored completely
 
     // Which of the two one-launch kernels runs is decided on the device (largest transition entry).
     if (MULTI && (a.maxmem[2] != 0) != P16) return;
@@ -503,6 +509,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
         published_count = 0;
         store_exit = 0;
         deps_ok = 0;
+        drained_b = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -787,7 +794,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             const int sbw = min(SB, S - sb0);
             int32_t* out = (a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice)
                            + (size_t)sb0 * m_pitch;
-            for (int row = lane; row < sbw; row += 32) {
+            for (int row = lane; row < sbw; row += 32 * NSW) {
                 const int mm = hdr0[row];
                 const int r = mm & 3;
                 const int g0 = m0 + mm - r;
@@ -803,7 +810,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
             bulk_commit();
             bulk_wait_read();                                     // the staging tile may be overwritten
             __syncwarp();
-            if (lane == 0) st_release_cta(&out_drained, it + 1);
+            if (lane == 0) red_release_cta_add(&out_drained, 1);
             if (publishing) {
                 // Hand the item to the publisher warp once its stores are complete.  Making them visible
                 // to the other SMs takes a fence, and a fence takes thousands of cycles while stores are
@@ -817,6 +824,13 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
                     }
                 }
                 bulk_wait_all();
+                if (NSW > 1) {
+                    WaitClock wc;                                 // the other store warp's rows are out as well
+                    while (ld_acquire_cta(&drained_b) < it + 1) {
+                        if (wc.expired()) { leave(true); return; }
+                        __nanosleep(100);
+                    }
+                }
                 {
                     WaitClock wc;                                 // the publisher reads item records: keep it close
                     while (it + 1 - *reinterpret_cast<volatile int*>(&published_count) > kPublishLag) {
@@ -831,6 +845,45 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
         bulk_wait_all();
         leave(false);
         return;
+    }
+
+    if (NSW > 1 && warp == NC + 4) {
+        // ------------------------------------------------------------ second store warp (packed path): rows lane+32, lane+96, ...
+        for (int it = 0;; ++it) {
+            if (!mbar_wait_idle(&out_full, it & 1)) {
+                if (lane == 0) atomicExch(a.err, 1);
+                return;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const int4 d = desc[it % kDescRing];
+            const int l = d.x, i = d.y;
+            if (l < 0) return;
+            const int m0 = d.z * TMB;
+            const int sb0 = d.w * SB;
+            const int sbw = min(SB, S - sb0);
+            int32_t* out = (a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice)
+                           + (size_t)sb0 * m_pitch;
+            for (int row = lane + 32; row < sbw; row += 64) {
+                const int mm = hdr0[row];
+                const int r = mm & 3;
+                const int g0 = m0 + mm - r;
+                const int hi = min(r + TMB, M + 1 - g0);
+                if (hi <= r) continue;
+                const int32_t* src = stg0 + row * RS;
+                int32_t* dst = out + (size_t)row * m_pitch + (size_t)g0;
+                const int lo4 = r ? 4 : 0, hi4 = hi & ~3;
+                if (hi4 > lo4) bulk_s2g(dst + lo4, src + lo4, (uint32_t)(hi4 - lo4) * 4u);
+                for (int x = r; x < min(lo4, hi); ++x) dst[x] = src[x];
+                for (int x = max(hi4, lo4); x < hi; ++x) dst[x] = src[x];
+            }
+            bulk_commit();
+            bulk_wait_read();
+            __syncwarp();
+            if (lane == 0) red_release_cta_add(&out_drained, 1);
+            bulk_wait_all();
+            __syncwarp();
+            if (lane == 0) st_release_cta(&drained_b, it + 1);
+        }
     }
 
     if (warp == NC + 3) {
@@ -879,7 +932,7 @@ __global__ void __launch_bounds__((NSG * NMS + 4) * 32, 1) layer_tiled_kernel(co
     // bounded wait until the store warp has read items 0 .. upto-1 out of the staging tile
     auto drained_wait = [&](int upto) -> bool {
         WaitClock wc;
-        while (ld_acquire_cta(&out_drained) < upto)
+        while (ld_acquire_cta(&out_drained) < upto * NSW)
             if (wc.expired()) return false;
         return true;
     };
@@ -1223,7 +1276,7 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
     if (packed) {
         // the packed 16-bit kernel over all layers: its own tensor maps (whole-tile boxes, packed trans rows)
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[2], (void*)&maps[3]};
-        return cudaLaunchCooperativeKernel((const void*)kern_packed, dim3(pl.grid), dim3((NSG * NMS + 4) * 32), args, (size_t)pl.p16_smem, st);
+        return cudaLaunchCooperativeKernel((const void*)kern_packed, dim3(pl.grid), dim3((NSG * NMS + 5) * 32), args, (size_t)pl.p16_smem, st);
     }
     if (l_last - l_first > 1) {
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[0], (void*)&maps[1]};
