@@ -210,8 +210,10 @@ def cost_model_scaled(torch, galv, hbm_gbs, barrier, copies=8192):
 
 def launches_per_step(w) -> int:
     # cost + trans kernels, validate + schedule + base layer, ONE cooperative launch over all layers,
-    # copy-last + finalize, backtrack
-    return (2 if w.has_model else 0) + 3 + 1 + 2 + 1
+    # copy-last + finalize, backtrack; where the shape allows the packed 16-bit path, the kernel that packs
+    # the trans rows and the launch of the other inner-loop variant (it returns at once) come on top
+    packable = w.S <= 64 and w.S % 4 == 0
+    return (2 if w.has_model else 0) + 3 + 1 + 2 + 1 + (2 if packable else 0)
 
 
 def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):
@@ -244,6 +246,7 @@ def main():
     ap.add_argument("--no-others", action="store_true", help="skip the side measurements of the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiler captures)")
+    ap.add_argument("--no-packed", action="store_true", help="keep the 32-bit inner loop where the packed 16-bit one would run")
     ap.add_argument("--batch", type=int, default=0, help="trim the workload to its first instances (profiler captures)")
     ap.add_argument("--layers", type=int, default=0, help="trim the workload to its first layers (profiler captures)")
     args = ap.parse_args()
@@ -281,7 +284,8 @@ def main():
     uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", "")
 
     with ClockSampler(uuid) as clk:
-        sb, r = bench_workload(torch, galv, w, args.steps, args.warmup, barrier)
+        sb, r = bench_workload(torch, galv, w, args.steps, args.warmup, barrier,
+                               flags=1 | (gb.KERNEL_NO_PACKED if args.no_packed else 0))
     t = max_over_ranks(r["seconds"])
     clocks = clk.summary()
     value = world * w.cells * args.steps / t
@@ -327,7 +331,8 @@ def main():
                      "traffic_unit": "bytes per launch (ncu dram read+write per layer x layers)",
                      "algorithmic_bytes_per_launch": 2 * 4 * w.B * w.S * w.m_pitch * (w.Lmax - 1),
                      "algorithmic_ops_per_launch": relax_per_launch,
-                     "kernel": "layer_tiled_kernel (one cooperative launch over all layers)",
+                     "kernel": "layer_tiled_kernel (one cooperative launch over all layers"
+                               + (", packed 16-bit variant)" if r["packed"] else ")"),
                      "launch_ms": r["layer_loop_ms"], "launch_ms_min": r["layer_loop_ms_min"],
                      "launch_ms_max": r["layer_loop_ms_max"], "launches_timed": r["layer_loop_launches_timed"],
                      "peak_source": "derived: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min per lane per clock"
@@ -365,6 +370,15 @@ def main():
         line["opt_cost_sum"] = r["opt_cost_sum"]
         del sbs
         torch.cuda.empty_cache()
+        if r["packed"]:
+            # the same step with the 32-bit inner loop (one relaxation per instruction), against its own peak
+            sb3, r3 = bench_workload(torch, galv, w, max(5, args.steps // 2), 3, barrier, flags=1 | gb.KERNEL_NO_PACKED)
+            line["inner_loop_32bit"] = {"ms_per_step": r3["ms_per_step"], "cells_per_s": r3["cells_per_s"],
+                                        "launch_ms": r3["layer_loop_ms"], "opt_cost_sum": r3["opt_cost_sum"],
+                                        "alu_frac": w.relaxations / (r3["layer_loop_ms"] * 1e-3) / 1e9 / ALU_PEAK_GOPS,
+                                        "peak": ALU_PEAK_GOPS}
+            del sb3
+            torch.cuda.empty_cache()
         # Cost-only search: no table kept, two layers roll in the workspace (optimum per instance, no plan).
         # All the relaxations are done; the tables' HBM footprint is 2 layers instead of Lmax.
         sbc, rc = bench_workload(torch, galv, w, max(5, args.steps // 2), 3, barrier, flags=0)

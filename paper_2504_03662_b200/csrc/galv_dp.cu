@@ -977,20 +977,28 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
                     const int32_t* rp = raw0 + (c / BOXC) * (S * BOXC) + (c % BOXC) + h * rows * BOXC;
                     int v[32];
                     int mn = kInf;
+                    if (rows == 32) {                           // S = 64: no row guards
 #pragma unroll
-                    for (int r = 0; r < 32; ++r) {
-                        v[r] = r < rows ? rp[r * BOXC] : kInf;
-                        mn = min(mn, v[r]);
+                        for (int r = 0; r < 32; ++r) {
+                            v[r] = rp[r * BOXC];
+                            mn = min(mn, v[r]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int r = 0; r < 32; ++r) {
+                            v[r] = r < rows ? rp[r * BOXC] : kInf;
+                            mn = min(mn, v[r]);
+                        }
                     }
                     mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, LPC));
                     if (cg < cend) {
                         uint32_t* out = pkc + (h * (rows / 2)) * TMB + c;
 #pragma unroll
                         for (int q = 0; q < 16; ++q)
-                            if (2 * q < rows) {
-                                const int d0 = __viaddmin_s32(v[2 * q], -mn, K);
-                                const int d1 = __viaddmin_s32(v[2 * q + 1], -mn, K);
-                                out[q * TMB] = (uint32_t)d0 | ((uint32_t)d1 << 16);
+                            if (rows == 32 || 2 * q < rows) {
+                                const uint32_t d0 = (uint32_t)__viaddmin_s32(v[2 * q], -mn, K);
+                                const uint32_t d1 = (uint32_t)__viaddmin_s32(v[2 * q + 1], -mn, K);
+                                out[q * TMB] = __byte_perm(d0, d1, 0x5410);      // d0 | d1 << 16
                             }
                         if (h == 0) basep[c] = mn;
                     }
