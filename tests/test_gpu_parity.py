@@ -485,3 +485,27 @@ def test_packed_16bit_path_choice_and_parity(orc, galv, S, M, B, Lmax):
         sb = SearchBuffers(galv, w, flags)
         sb.dp_search()
         assert not galv.galv_dp_search_path(sb.shape, sb.workspace)
+
+
+def test_packed_path_with_costs_near_the_limit(orc, galv):
+    """Path sums just below 2^30 (the validation bound), tiny transitions: the packed loop works on differences,
+    so the size of the costs themselves must not matter; a column without any finite value stays +inf."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    B, Lmax, S, M = 3, 4, 16, 700
+    w = inputs.random_tables(123, B, Lmax, S, M, mem_lo=0, mem_hi=200, time_hi=1000, trans_hi=9)
+    w.time_q[:, :, :] += (2 ** 30 - 1 - 4 * 1000 - 3 * 9) // 4 - 1     # four layers: the worst path sum stays just below 2^30 - 1
+    w.time_q[1, 2, ::2] = 0                                              # and some spread between strategies
+    w.mem_q[2, 1, :] = M + 1                                             # instance 2: nothing fits from layer 1 on
+    assert orc.validate(w.time_q[0], w.mem_q[0], w.trans_q[0]) == 0
+    sb = SearchBuffers(galv, w, gb.STORE_C_FULL)
+    sb.dp_search(); sb.backtrack()
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace)
+    res = sb.results()
+    for i in range(B):
+        r = orc.search(w.time_q[i], w.mem_q[i], w.trans_q[i], M)
+        assert res["status"][i] == r["status"] and res["opt_cost"][i] == r["opt_cost"], i
+        assert (res["plan"][i] == r["plan"]).all()
+        assert (sb.table(i) == r["C"]).all(), i
+    assert res["status"][2] == 1 and res["opt_cost"][2] == INF
