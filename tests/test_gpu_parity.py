@@ -509,3 +509,28 @@ def test_packed_path_with_costs_near_the_limit(orc, galv):
         assert (res["plan"][i] == r["plan"]).all()
         assert (sb.table(i) == r["C"]).all(), i
     assert res["status"][2] == 1 and res["opt_cost"][2] == INF
+
+
+def test_two_streams_at_once(orc, galv):
+    """Two searches enqueued on two streams, each with its own workspace: the one-launch kernels take turns on
+    the GPU (a cooperative launch needs all its CTAs resident); both must finish and be right."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    wa = inputs.random_tables(501, 40, 20, 32, 2000, mem_lo=1, mem_hi=150, trans_hi=900)       # packed loop
+    wb = inputs.random_tables(502, 30, 25, 24, 1500, mem_lo=1, mem_hi=100, trans_hi=60000)     # 32-bit loop
+    sa, sb_ = SearchBuffers(galv, wa, gb.STORE_C_FULL), SearchBuffers(galv, wb, gb.STORE_C_FULL)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        with torch.cuda.stream(s1):
+            sa.dp_search(); sa.backtrack()
+        with torch.cuda.stream(s2):
+            sb_.dp_search(); sb_.backtrack()
+    torch.cuda.synchronize()
+    for w, s in ((wa, sa), (wb, sb_)):
+        res = s.results()
+        for i in range(0, w.B, 7):
+            r = orc.search(w.time_q[i], w.mem_q[i], w.trans_q[i], w.M)
+            assert res["status"][i] == r["status"] and res["opt_cost"][i] == r["opt_cost"]
+            assert (res["plan"][i] == r["plan"]).all() and (s.table(i) == r["C"]).all()
