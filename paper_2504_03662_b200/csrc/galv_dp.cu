@@ -1042,8 +1042,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
                         pt += KQ * SB;
                     }
                 };
-                steps(std::integral_constant<int, 16>());
-                steps(std::integral_constant<int, 4>());
+                steps(std::integral_constant<int, 8>());
                 steps(std::integral_constant<int, 1>());
             }
             int mm[TS], tt[TS];
