@@ -979,9 +979,10 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
                     int mn = kInf;
                     if (rows == 32) {                           // S = 64: no row guards
 #pragma unroll
-                        for (int r = 0; r < 32; ++r) {
+                        for (int r = 0; r < 32; r += 2) {
                             v[r] = rp[r * BOXC];
-                            mn = min(mn, v[r]);
+                            v[r + 1] = rp[(r + 1) * BOXC];
+                            mn = __vimin3_s32(mn, v[r], v[r + 1]);
                         }
                     } else {
 #pragma unroll
@@ -1071,7 +1072,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
                     for (int j = 0; j < TM; ++j)
                         if (j < nj) {
                             const uint32_t x = (uint32_t)acc[j][u];
-                            const int w = (int)min(x & 0xffffu, x >> 16);         // the better of the two row parities
+                            const int w = (int)__vminu2(x, x >> 16);                // the better of the two row parities (upper half: min with 0)
                             const int v = __viaddmin_s32(bs[j], w, kInf);          // back on the column's base (+inf stays)
                             R[j * 32] = __viaddmin_s32(v, tt[u], kInf);
                         }
