@@ -371,6 +371,19 @@ def main():
         del sbs
         torch.cuda.empty_cache()
         if r["packed"]:
+            # The same step with GALV_SKIP_DOMINATED (and with both flags): row pairs that cannot win in any
+            # column of a tile are left out of the inner loop.  Same tables; how much is left out depends on the
+            # spread of the costs, so it stands beside the headline, which does all the relaxations.
+            for key, fl in (("with_dominated_rows_skipped", gb.SKIP_DOMINATED), ("with_both_skips", gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE)):
+                sbd, rd = bench_workload(torch, galv, w, max(5, args.steps // 2), 3, barrier, flags=1 | fl)
+                line[key] = {"ms_per_step": rd["ms_per_step"], "cells_per_s": rd["cells_per_s"],
+                             "searches_per_s": rd["searches_per_s"], "opt_cost_sum": rd["opt_cost_sum"],
+                             "launch_ms": rd["layer_loop_ms"],
+                             "hbm_frac": hbm_bytes / (rd["layer_loop_ms"] * 1e-3) / (hbm_gbs * 1e9),
+                             "note": "part of the relaxations is proved unnecessary and left out: no ALU-roofline fraction"}
+                del sbd
+                torch.cuda.empty_cache()
+        if r["packed"]:
             # the same step with the 32-bit inner loop (one relaxation per instruction), against its own peak
             sb3, r3 = bench_workload(torch, galv, w, max(5, args.steps // 2), 3, barrier, flags=1 | gb.KERNEL_NO_PACKED)
             line["inner_loop_32bit"] = {"ms_per_step": r3["ms_per_step"], "cells_per_s": r3["cells_per_s"],

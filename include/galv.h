@@ -72,6 +72,10 @@ extern "C" {
 #define GALV_SKIP_INFEASIBLE 1024 /* tiles wholly below the previous layer's feasibility frontier (sum of the
                                      layers' smallest mem) read only +inf: write their +inf results without
                                      loading or relaxing anything.  Same tables, less work on tight budgets. */
+#define GALV_SKIP_DOMINATED 8192 /* packed 16-bit path only (ignored elsewhere): a candidate more than the largest
+                                    transition entry above its column's best previous-layer value cannot win or tie;
+                                    row pairs that are such in all 128 columns of a warp group's tile are left out of
+                                    the inner loop.  Same tables; the work then depends on the spread of the costs. */
 
 typedef struct galv_ctx galv_ctx;
 

@@ -17,6 +17,7 @@ INF = 2 ** 30 - 1
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 STATUS_INFEASIBLE, STATUS_BAD_INPUT, STATUS_OVERFLOW_RISK, STATUS_TIMEOUT = 1, 2, 4, 8
 STORE_C_FULL, STORE_ARGMIN, KERNEL_REFERENCE, KERNEL_PER_LAYER, SKIP_INFEASIBLE = 1, 2, 256, 512, 1024
+SKIP_DOMINATED = 8192
 DEBUG_WITHHOLD_LOAD = 2048
 KERNEL_NO_PACKED = 4096
 TRANS_PER_LAYER = 4

@@ -437,7 +437,7 @@ constexpr int kDescRing = 16;
 // is rounded, clamped candidates stay above every possible winner.  The whole tile (all S rows) comes from
 // the table as int32 into ONE buffer and is rebased by the consumer warps into one of two packed stages, so
 // the next tile's load runs under this tile's inner loop.
-template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false>
+template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false, bool DOM = false>
 __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
                                                                               const __grid_constant__ CUtensorMap map_t)
@@ -488,11 +488,11 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
 
     // stage: NBOX boxes of [KS][BOXC] previous-layer values, then [KS][SB] trans values; 128-byte multiples.
     // Packed path: the raw tile (NBOX boxes of [S][BOXC]) first, then two stages of [Q][TMB] packed values,
-    // [Q][SB] packed trans entries and [TMB] column bases.
+    // [Q][SB] packed trans entries, [TMB] column bases and one word per consumer warp (row pairs alive in its columns).
     int32_t* const raw0 = reinterpret_cast<int32_t*>(smem_raw);
     const int raw_elems = P16 ? ((S * TMB + 31) & ~31) : 0;
     int32_t* const stage0 = raw0 + raw_elems;
-    const int stage_elems = P16 ? ((Q * TMB + Q * SB + TMB + 31) & ~31) : ((KS * (TMB + SB) + 31) & ~31);
+    const int stage_elems = P16 ? ((Q * TMB + Q * SB + TMB + NC + 31) & ~31) : ((KS * (TMB + SB) + 31) & ~31);
     int32_t* const meta0 = stage0 + NST * stage_elems;
     // staging tile [SB][RS] + its header: mem(l,s) per row, instance, last-layer flag
     int32_t* const stg0 = meta0 + ((NST * META + 31) & ~31);
@@ -943,6 +943,8 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
                                                            // each with half of the rows (S / 2 <= 32 values, in registers)
         const int K = a.maxmem[1] + 1;                     // a candidate this far above the column's best cannot win
         const int rows = S / 2;                            // S % 4 == 0: whole row pairs per lane
+        constexpr bool dom = DOM;                          // leave dominated row pairs out (an instantiation of its own:
+                                                           // the extra code costs the plain packed loop 4 %)
         for (int it = 0;; ++it) {
             const int st = it & 1;
             if (!mbar_wait(&full_bar[st], (it >> 1) & 1)) {
@@ -965,12 +967,15 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
             uint32_t* const pkc = reinterpret_cast<uint32_t*>(stg);
             const uint32_t* const pkt = reinterpret_cast<const uint32_t*>(stg + Q * TMB);
             int32_t* const basep = stg + Q * TMB + Q * SB;
+            uint32_t* const alivep = reinterpret_cast<uint32_t*>(basep + TMB);
             const int32_t* const meta = meta0 + st * META;
             const bool skipped = meta[2 * SB + 1] != 0;     // nothing but +inf to read: no data was loaded
             if (!skipped) {
                 // rebase: this warp's share of the group's columns, every row of them, read once
                 const int cl = lane % LPC, h = lane / LPC;
                 const int cend = min(sg * CW + CW, 32 * TM);
+                const uint32_t kk = (uint32_t)K * 0x10001u;     // a pair of clamped values: neither row can win in this column
+                uint32_t alive = 0;                             // row pairs of this lane's half that can still win in its columns
                 for (int c0 = sg * CW; c0 < cend; c0 += LPC) {
                     const int cg = c0 + cl;                     // column inside the group
                     const int c = ms * (32 * TM) + min(cg, 32 * TM - 1);
@@ -994,15 +999,23 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
                     mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, LPC));
                     if (cg < cend) {
                         uint32_t* out = pkc + (h * (rows / 2)) * TMB + c;
+                        // columns past the budget and columns without a finite value produce nothing
+                        const bool track = dom && mn < kInf && mw + (c - ms * (32 * TM)) <= M;
 #pragma unroll
                         for (int q = 0; q < 16; ++q)
                             if (rows == 32 || 2 * q < rows) {
                                 const uint32_t d0 = (uint32_t)__viaddmin_s32(v[2 * q], -mn, K);
                                 const uint32_t d1 = (uint32_t)__viaddmin_s32(v[2 * q + 1], -mn, K);
-                                out[q * TMB] = __byte_perm(d0, d1, 0x5410);      // d0 | d1 << 16
+                                const uint32_t pk = __byte_perm(d0, d1, 0x5410);  // d0 | d1 << 16
+                                out[q * TMB] = pk;
+                                if (track && pk != kk) alive |= 1u << q;
                             }
                         if (h == 0) basep[c] = mn;
                     }
+                }
+                if (dom) {
+                    alive = __reduce_or_sync(0xffffffffu, alive << (h * (rows / 2)));
+                    if (lane == 0) alivep[ms * NSG + sg] = alive;
                 }
             }
             __syncwarp();
@@ -1043,8 +1056,32 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
                         pt += KQ * SB;
                     }
                 };
-                steps(std::integral_constant<int, 8>());
-                steps(std::integral_constant<int, 1>());
+                if (!dom) {
+                    steps(std::integral_constant<int, 8>());
+                    steps(std::integral_constant<int, 1>());
+                } else {
+                    // Dominated rows left out: a row pair whose values lie more than the largest transition entry
+                    // above the column's best in every column of this group cannot supply a minimum (not even a
+                    // tie), so only the pairs some warp of the group found alive are relaxed.  Same results.
+                    uint32_t live = 0;
+#pragma unroll
+                    for (int g = 0; g < NSG; ++g) live |= alivep[ms * NSG + g];
+                    while (live) {
+                        const int qq = __ffs(live) - 1;
+                        live &= live - 1;
+                        uint32_t c[TM];
+#pragma unroll
+                        for (int j = 0; j < TM; ++j) c[j] = pc[qq * TMB + j * 32];
+                        const uint4 t0 = *reinterpret_cast<const uint4*>(pt + qq * SB);
+                        const uint4 t1 = *reinterpret_cast<const uint4*>(pt + qq * SB + 4);
+                        const uint32_t t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                        for (int j = 0; j < TM; ++j)
+#pragma unroll
+                            for (int u = 0; u < TS; ++u)
+                                acc[j][u] = (int)__viaddmin_u16x2(c[j], t[u], (uint32_t)acc[j][u]);
+                    }
+                }
             }
             int mm[TS], tt[TS];
             {
@@ -1275,16 +1312,18 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
     auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG, false>;
     auto kern_multi = layer_tiled_kernel<TM, NSG, NMS, false, true>;
     auto kern_packed = layer_tiled_kernel<TM, NSG, NMS, false, true, true>;
+    auto kern_packed_dom = layer_tiled_kernel<TM, NSG, NMS, false, true, true, true>;
     if (!maps) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_multi, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+        if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed_dom, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         return e;
     }
     if (packed) {
         // the packed 16-bit kernel over all layers: its own tensor maps (whole-tile boxes, packed trans rows)
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[2], (void*)&maps[3]};
-        return cudaLaunchCooperativeKernel((const void*)kern_packed, dim3(pl.grid), dim3((NSG * NMS + 5) * 32), args, (size_t)pl.p16_smem, st);
+        return cudaLaunchCooperativeKernel(a.skip_dom ? (const void*)kern_packed_dom : (const void*)kern_packed, dim3(pl.grid), dim3((NSG * NMS + 5) * 32), args, (size_t)pl.p16_smem, st);
     }
     if (l_last - l_first > 1) {
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[0], (void*)&maps[1]};
@@ -1386,7 +1425,7 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     {
         const int q = S / 2;
         const int raw = (S * pl->tmb * 4 + 127) & ~127;
-        const int pst = ((q * pl->tmb + q * pl->sb + pl->tmb) * 4 + 127) & ~127;
+        const int pst = ((q * pl->tmb + q * pl->sb + pl->tmb + pl->nsg * pl->nms) * 4 + 127) & ~127;
         const int total = raw + 2 * pst + ((2 * (2 * pl->sb + 4) + 31) & ~31) * 4 + staging;
         pl->p16 = S <= 64 && S % 4 == 0 && pl->nsb == 1 && !(sh->flags & GALV_STORE_ARGMIN) && total <= budget;
         pl->p16_smem = total;
@@ -1496,6 +1535,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     }
     DpArgs ap = a;
     ap.withhold = (sh->flags & GALV_DEBUG_WITHHOLD_LOAD) != 0;
+    ap.skip_dom = (sh->flags & GALV_SKIP_DOMINATED) != 0;
     if (!(sh->flags & GALV_SKIP_INFEASIBLE)) ap.front = nullptr;
     ap.tile_done = nullptr;
     ap.maxmem = a.err + 1;

@@ -64,6 +64,7 @@ struct DpArgs {
     int32_t* tcount;     // [Lmax][ntiles_m] layers 1..l whose items include tile t
     int32_t* status;
     int withhold;        // test hook: CTA 0 never loads its first chunk, so that the bounded waits run out
+    int skip_dom;        // packed path: leave out row pairs that cannot win in any column of a warp group's tile
 };
 
 // records `text` as the context's last error and returns `code`

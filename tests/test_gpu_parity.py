@@ -194,7 +194,7 @@ def test_config4_full_size(orc, galv):
     assert (res2["opt_cost"] == res["opt_cost"]).all() and (res2["plan"] == res["plan"]).all()
 
 
-@pytest.mark.parametrize("flags", [1, 1 | 1024])      # plain; tiles below the feasibility frontier skipped
+@pytest.mark.parametrize("flags", [1, 1 | 1024, 1 | 8192, 1 | 1024 | 8192])      # plain; tiles below the feasibility frontier skipped; dominated rows left out; both
 def test_config3_full_size(orc, galv, flags):
     import torch
     w = inputs.config3()
@@ -472,9 +472,15 @@ def test_packed_16bit_path_choice_and_parity(orc, galv, S, M, B, Lmax):
         plain.dp_search(); plain.backtrack()
         assert not galv.galv_dp_search_path(plain.shape, plain.workspace)
         assert torch.equal(sb.status, plain.status) and torch.equal(sb.opt_cost, plain.opt_cost)
+        pruned = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.SKIP_DOMINATED)     # dominated row pairs left out
+        pruned.dp_search(); pruned.backtrack()
+        assert galv.galv_dp_search_path(pruned.shape, pruned.workspace) == want
+        assert torch.equal(pruned.status, plain.status) and torch.equal(pruned.opt_cost, plain.opt_cost)
+        assert torch.equal(pruned.plan, plain.plan)
         for i in range(B):
             Li = int(w.L[i])
             assert torch.equal(sb.C[i, :Li], plain.C[i, :Li]), (top, i)
+            assert torch.equal(pruned.C[i, :Li], plain.C[i, :Li]), (top, i)
             r = orc.search(w.time_q[i, :Li], w.mem_q[i, :Li], w.trans_q[i], M)
             assert res["status"][i] == r["status"] and res["opt_cost"][i] == r["opt_cost"]
             if r["C"] is not None:
@@ -485,6 +491,34 @@ def test_packed_16bit_path_choice_and_parity(orc, galv, S, M, B, Lmax):
         sb = SearchBuffers(galv, w, flags)
         sb.dp_search()
         assert not galv.galv_dp_search_path(sb.shape, sb.workspace)
+
+
+@pytest.mark.parametrize("S,M,trans_hi,time_hi", [(4, 300, 0, 50), (16, 1000, 1, 1000), (36, 515, 40, 100000),
+                                                 (64, 2100, 500, 20), (64, 767, 32767, 10 ** 6), (8, 255, 3, 3)])
+def test_dominated_rows_left_out(orc, galv, S, M, trans_hi, time_hi):
+    """GALV_SKIP_DOMINATED: rows that cannot win in any column of a tile are not relaxed; the tables stay those of
+    the oracle when all transitions are 0 (only exact ties survive), with wide and with narrow spreads of the
+    costs, with columns that hold no finite value, and in the ragged last tile."""
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    B, Lmax = 5, 6
+    w = inputs.random_tables(9000 + S + trans_hi, B, Lmax, S, M, ragged=True, mem_lo=0, mem_hi=max(1, M // 3),
+                             time_hi=time_hi, trans_hi=trans_hi)
+    w.time_q[1, :, :] = 11                                       # one instance without any spread: every row ties
+    w.mem_q[2, 1, : max(1, S // 2)] = M + 9                      # rows that are +inf everywhere
+    w.mem_q[3, 0, :] = M // 2                                    # the lower half of every later column is +inf
+    for flags in (gb.STORE_C_FULL | gb.SKIP_DOMINATED, gb.SKIP_DOMINATED, gb.STORE_C_FULL | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE):
+        sb = SearchBuffers(galv, w, flags)
+        sb.dp_search(); sb.backtrack()
+        assert galv.galv_dp_search_path(sb.shape, sb.workspace)
+        res = sb.results()
+        for i in range(B):
+            Li = int(w.L[i])
+            r = orc.search(w.time_q[i, :Li], w.mem_q[i, :Li], w.trans_q[i], M)
+            assert res["status"][i] == r["status"] and res["opt_cost"][i] == r["opt_cost"], (flags, i)
+            if flags & gb.STORE_C_FULL:
+                assert (res["plan"][i, :Li] == r["plan"]).all(), (flags, i)
+                assert (sb.table(i)[:Li] == r["C"]).all(), (flags, i)
 
 
 def test_packed_path_with_costs_near_the_limit(orc, galv):
