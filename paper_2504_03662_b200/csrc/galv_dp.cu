@@ -438,7 +438,7 @@ constexpr int kDescRing = 16;
 // the table as int32 into ONE buffer and is rebased by the consumer warps into one of two packed stages, so
 // the next tile's load runs under this tile's inner loop.
 template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false, bool DOM = false>
-__global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
+__global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
                                                                               const __grid_constant__ CUtensorMap map_t)
 {
@@ -450,8 +450,11 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
     constexpr int META = 2 * SB + 4;
     constexpr int RS = TMB + 4;                           // staging row: TMB columns + room for the shift
     constexpr int KU = ARG ? 4 : 16;                      // k-steps per trip of the inner loop
-    constexpr int NSW = P16 ? 2 : 1;                      // store warps: the packed path's items are short enough for one
-                                                          // warp's row-by-row issue (about 10k cycles a tile) to hold them up
+    constexpr int NSW = P16 ? (DOM ? 4 : 2) : 1;          // store warps: the packed path's items are short enough for one
+                                                          // warp's row-by-row issue (about 10k cycles a tile) to hold them up;
+                                                          // with dominated rows left out the drain of the staging tile is
+                                                          // what the next tile waits for
+    constexpr int RPW = 64 / NSW;                         // staging rows (of at most 64) per store warp
     static_assert(TMB % BOXC == 0 && BOXC % (32 * TM) == 0, "a warp's columns must sit inside one box");
     static_assert(!(ARG && P16) && (!P16 || MULTI), "the packed path keeps no argmin and runs all layers in one launch");
 
@@ -468,7 +471,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
     __shared__ int store_exit;                             // the store warp has left
     __shared__ int deps_ok;                                // rolling buffer: items whose dependency wait the producer has passed
     __shared__ __align__(8) uint64_t conv_bar[16];         // packed path: the warps of a column group have rebased their columns
-    __shared__ int drained_b;                              // second store warp -> first: items whose rows it has stored completely
+    __shared__ int drained_b;                              // further store warps -> first: items whose rows they have stored completely (one count each)
 
     // Which of the two one-launch kernels runs is decided on the device (largest transition entry).
     if (MULTI && (a.maxmem[2] != 0) != P16) return;
@@ -794,7 +797,8 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
             const int sbw = min(SB, S - sb0);
             int32_t* out = (a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice)
                            + (size_t)sb0 * m_pitch;
-            for (int row = lane; row < sbw; row += 32 * NSW) {
+            // store warp w takes rows w * RPW .. (w + 1) * RPW - 1 (with two warps: rows lane and lane + 32)
+            for (int row = lane; row < (NSW <= 2 ? sbw : min(sbw, RPW)); row += (NSW <= 2 ? 32 * NSW : 32)) {
                 const int mm = hdr0[row];
                 const int r = mm & 3;
                 const int g0 = m0 + mm - r;
@@ -826,7 +830,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
                 bulk_wait_all();
                 if (NSW > 1) {
                     WaitClock wc;                                 // the other store warp's rows are out as well
-                    while (ld_acquire_cta(&drained_b) < it + 1) {
+                    while (ld_acquire_cta(&drained_b) < (it + 1) * (NSW - 1)) {
                         if (wc.expired()) { leave(true); return; }
                         __nanosleep(100);
                     }
@@ -847,8 +851,9 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
         return;
     }
 
-    if (NSW > 1 && warp == NC + 4) {
-        // ------------------------------------------------------------ second store warp (packed path): rows lane+32, lane+96, ...
+    if (NSW > 1 && (NSW == 2 ? warp == NC + 4 : warp >= NC + 4)) {
+        // ------------------------------------------------------------ further store warps (packed path)
+        const int sw = warp - (NC + 4) + 1;
         for (int it = 0;; ++it) {
             if (!mbar_wait_idle(&out_full, it & 1)) {
                 if (lane == 0) atomicExch(a.err, 1);
@@ -863,7 +868,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
             const int sbw = min(SB, S - sb0);
             int32_t* out = (a.C ? a.C + ((size_t)i * a.Lmax + l) * slice : a.roll + ((size_t)(l & 1) * a.B + i) * slice)
                            + (size_t)sb0 * m_pitch;
-            for (int row = lane + 32; row < sbw; row += 64) {
+            for (int row = (NSW == 2 ? lane + 32 : sw * RPW + lane); row < (NSW == 2 ? sbw : min(sbw, (sw + 1) * RPW)); row += (NSW == 2 ? 64 : 32)) {
                 const int mm = hdr0[row];
                 const int r = mm & 3;
                 const int g0 = m0 + mm - r;
@@ -882,7 +887,10 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? 5 : 4)) * 32, 1) layer_til
             if (lane == 0) red_release_cta_add(&out_drained, 1);
             bulk_wait_all();
             __syncwarp();
-            if (lane == 0) st_release_cta(&drained_b, it + 1);
+            if (lane == 0) {
+                if (NSW == 2) st_release_cta(&drained_b, it + 1);
+                else red_release_cta_add(&drained_b, 1);
+            }
         }
     }
 
@@ -1323,7 +1331,7 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
     if (packed) {
         // the packed 16-bit kernel over all layers: its own tensor maps (whole-tile boxes, packed trans rows)
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[2], (void*)&maps[3]};
-        return cudaLaunchCooperativeKernel(a.skip_dom ? (const void*)kern_packed_dom : (const void*)kern_packed, dim3(pl.grid), dim3((NSG * NMS + 5) * 32), args, (size_t)pl.p16_smem, st);
+        return cudaLaunchCooperativeKernel(a.skip_dom ? (const void*)kern_packed_dom : (const void*)kern_packed, dim3(pl.grid), dim3((NSG * NMS + (a.skip_dom ? 7 : 5)) * 32), args, (size_t)pl.p16_smem, st);
     }
     if (l_last - l_first > 1) {
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[0], (void*)&maps[1]};
