@@ -247,6 +247,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiler captures)")
     ap.add_argument("--no-packed", action="store_true", help="keep the 32-bit inner loop where the packed 16-bit one would run")
+    ap.add_argument("--skip-dominated", action="store_true", help="run with GALV_SKIP_DOMINATED (profiler captures; the roofline keys then do not apply)")
     ap.add_argument("--batch", type=int, default=0, help="trim the workload to its first instances (profiler captures)")
     ap.add_argument("--layers", type=int, default=0, help="trim the workload to its first layers (profiler captures)")
     args = ap.parse_args()
@@ -285,7 +286,7 @@ def main():
 
     with ClockSampler(uuid) as clk:
         sb, r = bench_workload(torch, galv, w, args.steps, args.warmup, barrier,
-                               flags=1 | (gb.KERNEL_NO_PACKED if args.no_packed else 0))
+                               flags=1 | (gb.KERNEL_NO_PACKED if args.no_packed else 0) | (gb.SKIP_DOMINATED if args.skip_dominated else 0))
     t = max_over_ranks(r["seconds"])
     clocks = clk.summary()
     value = world * w.cells * args.steps / t
