@@ -72,10 +72,12 @@ extern "C" {
 #define GALV_SKIP_INFEASIBLE 1024 /* tiles wholly below the previous layer's feasibility frontier (sum of the
                                      layers' smallest mem) read only +inf: write their +inf results without
                                      loading or relaxing anything.  Same tables, less work on tight budgets. */
-#define GALV_SKIP_DOMINATED 8192 /* packed 16-bit path only (ignored elsewhere): a candidate more than the largest
-                                    transition entry above its column's best previous-layer value cannot win or tie;
-                                    row pairs that are such in all 128 columns of a warp group's tile are left out of
-                                    the inner loop.  Same tables; the work then depends on the spread of the costs. */
+#define GALV_SKIP_DOMINATED 8192 /* a candidate more than the largest transition entry above its column's best
+                                    previous-layer value cannot win or tie; rows (row pairs in the packed loop) that
+                                    are such in all 128 columns of a warp group's tile are left out of the inner
+                                    loop.  Same tables; the work then depends on the spread of the costs.  Honoured
+                                    by the one-launch kernels without argmin table when S <= 64 (and, in the 32-bit
+                                    loop, a tile's S rows fit one stage); ignored elsewhere. */
 
 typedef struct galv_ctx galv_ctx;
 

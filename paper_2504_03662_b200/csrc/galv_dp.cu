@@ -447,7 +447,9 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
     constexpr int TMB = NMS * 32 * TM;                    // columns per item
     constexpr int BOXC = 32 * TM * ((NMS % 2 == 0 && 64 * TM <= 256) ? 2 : 1);   // columns per TMA box (box extents are <= 256)
     constexpr int NBOX = TMB / BOXC;
-    constexpr int META = 2 * SB + 4;
+    constexpr int META = 2 * SB + 4 + ((DOM && !P16) ? ((2 * NMS + 3) & ~3) : 0);   // 32-bit loop without dominated rows: two words of live rows per
+                                                                                    // column group; a multiple of 4 (the record is read 16 bytes at a time)
+    static_assert(META % 4 == 0, "item records are read with 16-byte loads");
     constexpr int RS = TMB + 4;                           // staging row: TMB columns + room for the shift
     constexpr int KU = ARG ? 4 : 16;                      // k-steps per trip of the inner loop
     constexpr int NSW = P16 ? (DOM ? 4 : 2) : 1;          // store warps: the packed path's items are short enough for one
@@ -726,6 +728,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                     if (lane == 0) meta[2 * SB] = i;
                 }
                 if (lane == 0) meta[2 * SB + 1] = skip;           // the consumers leave this chunk's k-steps out
+                if (DOM && !P16 && lane < 2 * NMS) meta[2 * SB + 4 + lane] = 0;   // live rows: the consumers OR into these
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&full_bar[st]);
             }
@@ -1177,56 +1180,119 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
             // this warp's columns inside their box, and its 8 trans columns
             const int32_t* cs = stage0 + st * stage_elems + ((ms * (32 * TM)) / BOXC) * (KS * BOXC) + (ms * (32 * TM)) % BOXC + lane;
             const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
-            if (nj == TM) {
-                // trips of KU k-steps, then of 4, then single ones: loop control and pointer bumps are ALU
-                // instructions too, one trip of 16 k-steps spends 4 of them on 512 relaxations
-                int k = 0;
-                auto steps = [&](auto ku) {
-                    constexpr int K = decltype(ku)::value;
-                    for (; k + K <= kn; k += K) {
+            if constexpr (DOM && !P16) {
+                // Dominated rows left out (one chunk per item, S <= 64: the host takes this instantiation only then).
+                // A candidate more than the largest transition entry above its column's best cannot win or tie;
+                // a row that is such in every column of this group's tile is not relaxed.  Each warp scans its
+                // share of the group's columns (minimum, then one compare per value), the group ORs the rows still
+                // alive into two words beside the item's record, and after a barrier walks their set bits.
+                uint32_t* const live_w = reinterpret_cast<uint32_t*>(meta0 + st * META + 2 * SB + 4 + 2 * ms);
+                if (kn > 0) {
+                    constexpr int CW = (32 * TM + NSG - 1) / NSG;   // columns of the group each of its warps scans
+                    const int kmax = a.maxmem[1];
+                    const int cend = min(sg * CW + CW, 32 * TM);
+                    uint32_t lo = 0, hi = 0;
+                    for (int c0 = sg * CW; c0 < cend; c0 += 32) {
+                        const int cg = c0 + lane;
+                        const int c = ms * (32 * TM) + min(cg, 32 * TM - 1);
+                        const int32_t* p = stage0 + st * stage_elems + (c / BOXC) * (KS * BOXC) + c % BOXC;
+                        int mn = kInf;
+#pragma unroll 4
+                        for (int r = 0; r < kn; ++r) mn = min(mn, p[r * BOXC]);
+                        // columns past the budget and columns without a finite value produce nothing
+                        if (cg < cend && mn < kInf && mw + cg <= M) {
+                            const int lim = mn + kmax;              // both below 2^30
+#pragma unroll 4
+                            for (int r = 0; r < min(kn, 32); ++r) lo |= (p[r * BOXC] <= lim) ? 1u << r : 0u;
+#pragma unroll 4
+                            for (int r = 32; r < kn; ++r) hi |= (p[r * BOXC] <= lim) ? 1u << (r - 32) : 0u;
+                        }
+                    }
+                    lo = __reduce_or_sync(0xffffffffu, lo);
+                    hi = __reduce_or_sync(0xffffffffu, hi);
+                    if (lane == 0) {
+                        if (lo) atomicOr(live_w, lo);
+                        if (hi) atomicOr(live_w + 1, hi);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&conv_bar[ms]);
+                if (!mbar_wait(&conv_bar[ms], it & 1)) {
+                    if (lane == 0) atomicExch(a.err, 1);
+                    return;
+                }
+                if (nj > 0 && kn > 0) {
 #pragma unroll
-                        for (int kk = 0; kk < K; ++kk) {
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t lv = *reinterpret_cast<volatile uint32_t*>(live_w + half);
+                        while (lv) {
+                            const int r = __ffs(lv) - 1 + 32 * half;
+                            lv &= lv - 1;
                             int c[TM];
 #pragma unroll
-                            for (int j = 0; j < TM; ++j) c[j] = cs[kk * BOXC + j * 32];
-                            const int4 t0 = *reinterpret_cast<const int4*>(ts + kk * SB);
-                            const int4 t1 = *reinterpret_cast<const int4*>(ts + kk * SB + 4);
+                            for (int j = 0; j < TM; ++j) c[j] = cs[r * BOXC + j * 32];
+                            const int4 t0 = *reinterpret_cast<const int4*>(ts + r * SB);
+                            const int4 t1 = *reinterpret_cast<const int4*>(ts + r * SB + 4);
                             const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
 #pragma unroll
                             for (int j = 0; j < TM; ++j)
 #pragma unroll
-                                for (int u = 0; u < TS; ++u) {
-                                    if (ARG) {
-                                        const int cand = c[j] + t[u];
-                                        if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k + kk; }
-                                    } else {
-                                        acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
-                                    }
-                                }
+                                for (int u = 0; u < TS; ++u) acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
                         }
-                        cs += K * BOXC;
-                        ts += K * SB;
                     }
-                };
-                steps(std::integral_constant<int, KU>());
-                steps(std::integral_constant<int, 4>());
-                steps(std::integral_constant<int, 1>());
-            } else if (nj > 0) {
-                // ragged last tile: only the first nj column groups carry work
-                for (int k = 0; k < kn; ++k) {
-                    const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
-                    const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
-                    const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-#pragma unroll
-                    for (int j = 0; j < TM; ++j)
-                        if (j < nj) {
-                            const int c = cs[k * BOXC + j * 32];
-#pragma unroll
-                            for (int u = 0; u < TS; ++u) {
-                                const int cand = c + t[u];
-                                if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
+                }
+            } else {
+                if (nj == TM) {
+                    // trips of KU k-steps, then of 4, then single ones: loop control and pointer bumps are ALU
+                    // instructions too, one trip of 16 k-steps spends 4 of them on 512 relaxations
+                    int k = 0;
+                    auto steps = [&](auto ku) {
+                        constexpr int K = decltype(ku)::value;
+                        for (; k + K <= kn; k += K) {
+    #pragma unroll
+                            for (int kk = 0; kk < K; ++kk) {
+                                int c[TM];
+    #pragma unroll
+                                for (int j = 0; j < TM; ++j) c[j] = cs[kk * BOXC + j * 32];
+                                const int4 t0 = *reinterpret_cast<const int4*>(ts + kk * SB);
+                                const int4 t1 = *reinterpret_cast<const int4*>(ts + kk * SB + 4);
+                                const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+    #pragma unroll
+                                for (int j = 0; j < TM; ++j)
+    #pragma unroll
+                                    for (int u = 0; u < TS; ++u) {
+                                        if (ARG) {
+                                            const int cand = c[j] + t[u];
+                                            if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k + kk; }
+                                        } else {
+                                            acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                                        }
+                                    }
                             }
+                            cs += K * BOXC;
+                            ts += K * SB;
                         }
+                    };
+                    steps(std::integral_constant<int, KU>());
+                    steps(std::integral_constant<int, 4>());
+                    steps(std::integral_constant<int, 1>());
+                } else if (nj > 0) {
+                    // ragged last tile: only the first nj column groups carry work
+                    for (int k = 0; k < kn; ++k) {
+                        const int4 t0 = *reinterpret_cast<const int4*>(ts + k * SB);
+                        const int4 t1 = *reinterpret_cast<const int4*>(ts + k * SB + 4);
+                        const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+    #pragma unroll
+                        for (int j = 0; j < TM; ++j)
+                            if (j < nj) {
+                                const int c = cs[k * BOXC + j * 32];
+    #pragma unroll
+                                for (int u = 0; u < TS; ++u) {
+                                    const int cand = c + t[u];
+                                    if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
+                                }
+                            }
+                    }
                 }
             }
             if (kc == NKC - 1) {
@@ -1321,11 +1387,13 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
     auto kern_multi = layer_tiled_kernel<TM, NSG, NMS, false, true>;
     auto kern_packed = layer_tiled_kernel<TM, NSG, NMS, false, true, true>;
     auto kern_packed_dom = layer_tiled_kernel<TM, NSG, NMS, false, true, true, true>;
+    auto kern_multi_dom = layer_tiled_kernel<TM, NSG, NMS, false, true, false, true>;
     if (!maps) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_multi, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed_dom, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+        if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_multi_dom, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         return e;
     }
     if (packed) {
@@ -1335,7 +1403,9 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
     }
     if (l_last - l_first > 1) {
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[0], (void*)&maps[1]};
-        return cudaLaunchCooperativeKernel((const void*)kern_multi, dim3(pl.grid), dim3((NSG * NMS + 4) * 32), args, (size_t)pl.smem, st);
+        // dominated rows are left out where all S <= 64 rows of a tile sit in one stage
+        const bool dom = a.skip_dom && pl.nkc == 1 && a.S <= 64;
+        return cudaLaunchCooperativeKernel(dom ? (const void*)kern_multi_dom : (const void*)kern_multi, dim3(pl.grid), dim3((NSG * NMS + 4) * 32), args, (size_t)pl.smem, st);
     }
     kern<<<pl.grid, (NSG * NMS + 4) * 32, pl.smem, st>>>(a, pl, l_first, l_last, maps[0], maps[1]);
     return cudaGetLastError();
@@ -1410,13 +1480,14 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     const int row = (pl->tmb + pl->sb) * 4;
     // chunks of s': as few per item as leave room for two stages (every chunk costs the consumers
     // a barrier hand-over), of equal size, multiples of 8 rows; then as many stages as fit
+    const int dom_words = (sh->flags & GALV_SKIP_DOMINATED) ? ((2 * pl->nms + 3) & ~3) : 0;   // live-row words per column group in each item record
     int nkc = 1, ks = S, stage_bytes = 0, nst = 0, extra = 0;
     for (;; ++nkc) {
         ks = (S + nkc - 1) / nkc;
         if (ks >= 8) ks = (ks + 7) & ~7;
         stage_bytes = (ks * row + 127) & ~127;
         for (nst = kMaxStages; nst >= 2; --nst) {
-            extra = ((nst * (2 * pl->sb + 4) + 31) & ~31) * 4 + staging;  // item records of the stages
+            extra = ((nst * (2 * pl->sb + 4 + dom_words) + 31) & ~31) * 4 + staging;  // item records of the stages
             if (nst * stage_bytes + extra <= budget) break;
         }
         if (nst >= 2 || ks == 1) break;

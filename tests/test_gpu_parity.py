@@ -194,6 +194,17 @@ def test_config4_full_size(orc, galv):
     assert (res2["opt_cost"] == res["opt_cost"]).all() and (res2["plan"] == res["plan"]).all()
 
 
+def test_config4_full_size_dominated_rows_skipped(orc, galv):
+    """The 32-bit loop (transition entries to 5e4) with dominated rows left out, all 1024 instances."""
+    from paper_2504_03662_b200 import binding as gb
+    w = inputs.config4()
+    idx = [0, 511, 1023] + list(range(100, 1024, 300))
+    sb, res = check_batch(orc, galv, w, gb.STORE_C_FULL | gb.SKIP_DOMINATED, idx=idx)
+    assert not galv.galv_dp_search_path(sb.shape, sb.workspace)
+    assert (res["status"] == 0).all()
+    _properties_all(orc, w, w.time_q, w.mem_q, w.trans_q, sb, res)
+
+
 @pytest.mark.parametrize("flags", [1, 1 | 1024, 1 | 8192, 1 | 1024 | 8192])      # plain; tiles below the feasibility frontier skipped; dominated rows left out; both
 def test_config3_full_size(orc, galv, flags):
     import torch
@@ -494,7 +505,8 @@ def test_packed_16bit_path_choice_and_parity(orc, galv, S, M, B, Lmax):
 
 
 @pytest.mark.parametrize("S,M,trans_hi,time_hi", [(4, 300, 0, 50), (16, 1000, 1, 1000), (36, 515, 40, 100000),
-                                                 (64, 2100, 500, 20), (64, 767, 32767, 10 ** 6), (8, 255, 3, 3)])
+                                                 (64, 2100, 500, 20), (64, 767, 32767, 10 ** 6), (8, 255, 3, 3),
+                                                 (32, 2100, 50000, 10 ** 6), (61, 700, 90000, 10 ** 5), (24, 130, 7, 10 ** 4)])
 def test_dominated_rows_left_out(orc, galv, S, M, trans_hi, time_hi):
     """GALV_SKIP_DOMINATED: rows that cannot win in any column of a tile are not relaxed; the tables stay those of
     the oracle when all transitions are 0 (only exact ties survive), with wide and with narrow spreads of the
@@ -507,10 +519,13 @@ def test_dominated_rows_left_out(orc, galv, S, M, trans_hi, time_hi):
     w.time_q[1, :, :] = 11                                       # one instance without any spread: every row ties
     w.mem_q[2, 1, : max(1, S // 2)] = M + 9                      # rows that are +inf everywhere
     w.mem_q[3, 0, :] = M // 2                                    # the lower half of every later column is +inf
-    for flags in (gb.STORE_C_FULL | gb.SKIP_DOMINATED, gb.SKIP_DOMINATED, gb.STORE_C_FULL | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE):
+    for flags in (gb.STORE_C_FULL | gb.SKIP_DOMINATED, gb.SKIP_DOMINATED, gb.STORE_C_FULL | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE,
+                  gb.STORE_C_FULL | gb.SKIP_DOMINATED | gb.KERNEL_NO_PACKED,            # the 32-bit loop's variant
+                  gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE | gb.KERNEL_NO_PACKED):
         sb = SearchBuffers(galv, w, flags)
         sb.dp_search(); sb.backtrack()
-        assert galv.galv_dp_search_path(sb.shape, sb.workspace)
+        packable = S % 4 == 0 and int(w.trans_q.max()) <= 32767 and not flags & gb.KERNEL_NO_PACKED
+        assert galv.galv_dp_search_path(sb.shape, sb.workspace) == packable
         res = sb.results()
         for i in range(B):
             Li = int(w.L[i])
