@@ -437,6 +437,29 @@ def test_cost_only_search_many_layers_against_full_table(galv):
             assert torch.equal(lean.C_last[ok], full.C_last[ok])
 
 
+@pytest.mark.parametrize("k", [3, 4])
+def test_skipping_flags_change_no_cell_of_the_large_workloads(galv, k):
+    """Every cell of every instance of configs 3 and 4: the tables, optima and plans with GALV_SKIP_DOMINATED |
+    GALV_SKIP_INFEASIBLE equal those of the plain run (which the exhaustive pass below ties to the oracle)."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    w = inputs.CONFIGS[k]()
+    plain = SearchBuffers(galv, w, gb.STORE_C_FULL)
+    plain.step()
+    skip = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE)
+    skip.step()
+    torch.cuda.synchronize()
+    assert torch.equal(plain.status, skip.status) and torch.equal(plain.opt_cost, skip.opt_cost)
+    assert torch.equal(plain.plan, skip.plan) and torch.equal(plain.mem_used, skip.mem_used)
+    M = w.M
+    for i in range(w.B):
+        Li = int(w.L[i])
+        assert torch.equal(plain.C[i, :Li, :, :M + 1], skip.C[i, :Li, :, :M + 1]), i
+    del plain, skip
+    torch.cuda.empty_cache()
+
+
 @pytest.mark.skipif(not os.environ.get("GALV_FULL_PARITY"), reason="every instance of the two large workloads: minutes; set GALV_FULL_PARITY=1")
 @pytest.mark.parametrize("k", [3, 4])
 def test_full_parity_every_instance(orc, galv, k):
