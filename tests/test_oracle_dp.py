@@ -143,6 +143,34 @@ def test_invariants(orc, seed):
             assert o == Ct[-1, budget].min() and p[-1] == int(Ct[-1, budget].argmin())
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_dominated_rows_never_supply_a_minimum(orc, seed):
+    """The argument behind GALV_SKIP_DOMINATED, checked on the oracle's own tables: a previous-layer entry more
+    than the largest transition entry above its column's best is never the argmin of any cell that reads the
+    column, and taking those entries out (setting them to +inf) changes no cell of the next layer."""
+    w = inputs.random_tables(700 + seed, 1, 7, 9, 120, mem_lo=0, mem_hi=35, time_hi=(5, 400, 100000)[seed % 3],
+                             trans_hi=(0, 3, 60, 2000)[seed % 4], dup_cols=(seed % 2 == 1))
+    t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
+    Ct, At = orc.dp(t, m, x, w.M)                               # [L][M+1][S]
+    tmax = int(x.max())
+    some_dominated = False
+    for l in range(1, 7):
+        prev = Ct[l - 1].astype(np.int64)
+        best = prev.min(axis=1, keepdims=True)
+        dominated = (prev - best > tmax) | (prev >= INF)          # per (column, strategy) of layer l-1
+        some_dominated |= bool((dominated & (prev < INF)).any())
+        pruned = np.where(dominated, INF, prev)
+        for s in range(9):
+            mem = int(m[l, s])
+            for mm in range(mem, w.M + 1):
+                a = int(At[l, mm, s])
+                if a != 255:
+                    assert not dominated[mm - mem, a], (l, mm, s)
+                cand = np.minimum(pruned[mm - mem] + x[:, s], INF)
+                assert min(int(cand.min()) + int(t[l, s]), INF) == Ct[l, mm, s], (l, mm, s)
+    assert some_dominated or seed % 3 == 0                      # the wide spreads really exercise it
+
+
 def test_single_strategy_closed_form(orc):
     w = inputs.random_tables(5, 1, 12, 1, 200, mem_lo=3, mem_hi=30)
     t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
