@@ -57,7 +57,7 @@ def test_equal_matrices_reduce_to_one(orc):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("flags", [1, 3, 2, 1 | 512])
+@pytest.mark.parametrize("flags", [1, 3, 2, 1 | 512, 1 | 8192 | 1024, 1 | 8192 | 4096])      # the last two: skipping flags, packed and 32-bit loop
 def test_gpu_parity(orc, flags):
     import torch
     from paper_2504_03662_b200 import binding as gb
