@@ -981,6 +981,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
             uint32_t* const alivep = reinterpret_cast<uint32_t*>(basep + TMB);
             const int32_t* const meta = meta0 + st * META;
             const bool skipped = meta[2 * SB + 1] != 0;     // nothing but +inf to read: no data was loaded
+            bool raw_released = false;
             if (!skipped) {
                 // rebase: this warp's share of the group's columns, every row of them, read once
                 const int cl = lane % LPC, h = lane / LPC;
@@ -1008,6 +1009,14 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                         }
                     }
                     mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, LPC));
+                    if (dom && c0 + LPC >= cend) {
+                        // last pass: every value this warp needs is in registers (the minimum has consumed them all),
+                        // so the raw buffer goes back before the packing: with the inner loop this short the next
+                        // tile's load latency is what the item waits for
+                        raw_released = true;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&empty_bar[0]);
+                    }
                     if (cg < cend) {
                         uint32_t* out = pkc + (h * (rows / 2)) * TMB + c;
                         // columns past the budget and columns without a finite value produce nothing
@@ -1031,7 +1040,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
             }
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&empty_bar[0]);                 // this warp is done with the raw tile
+                if (!raw_released) mbar_arrive(&empty_bar[0]);   // this warp is done with the raw tile
                 mbar_arrive(&conv_bar[ms]);                 // and its columns are there for the group
             }
             if (!mbar_wait(&conv_bar[ms], it & 1)) {
