@@ -317,7 +317,7 @@ def test_layers_with_different_tile_counts(orc, galv, flags):
     check_batch(orc, galv, w, flags)
 
 
-@pytest.mark.parametrize("flags", [1, 1 | 512])
+@pytest.mark.parametrize("flags", [1, 1 | 512, 1 | 8192, 1 | 8192 | 4096])     # one launch, per layer, dominated rows skipped (packed, 32-bit)
 def test_bounded_waits_run_out_cleanly(orc, galv, flags):
     """A stage that never fills: the waits give up, the status says TIMEOUT, the context keeps working."""
     import time
@@ -357,7 +357,7 @@ def test_one_launch_against_reference_kernel_on_many_shapes(galv, block):
             w.mem_q[:, int(rng.integers(1, Lmax)), :] += M // 2       # one heavy layer: fewer tiles there
         ref = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_REFERENCE)
         ref.dp_search()
-        one = SearchBuffers(galv, w, gb.STORE_C_FULL | (gb.SKIP_INFEASIBLE if case % 3 == 2 else 0))
+        one = SearchBuffers(galv, w, gb.STORE_C_FULL | (gb.SKIP_INFEASIBLE if case % 3 == 2 else 0) | (gb.SKIP_DOMINATED if case % 4 == 1 else 0))
         for _ in range(2):
             one.C.fill_(-7)
             one.dp_search()
