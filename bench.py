@@ -349,7 +349,7 @@ def main():
         # HBM side of the roofline: every table cell written once and read once by the next layer
         from paper_2504_03662_b200.binding import make_shape
         pitch = make_shape(w.B, w.Lmax, w.S, w.M).m_pitch
-        hbm_bytes = 2 * 4 * w.B * w.Lmax * w.S * pitch
+        hbm_bytes = 2 * 4 * int(np.sum(w.L)) * w.S * pitch
         peaks = {}
         try:
             peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -411,13 +411,13 @@ def main():
             o = {key: rk[key] for key in ("ms_per_step", "cells_per_s", "relax_per_s", "searches_per_s")}
             o["alu_frac"] = rk["relax_per_s"] / (ALU_PEAK_GOPS * 1e9 * (2 if rk["packed"] else 1))
             o["packed"] = rk["packed"]
-            if k == 4:
+            if k in (1, 2, 4):
                 # with both opt-in flags (work proved unnecessary left out; same tables): no ALU-roofline fraction
                 sbd, rd = bench_workload(torch, galv, wk, max(5, args.steps // 2), 3, barrier,
                                          flags=1 | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE)
                 pitch4 = make_shape(wk.B, wk.Lmax, wk.S, wk.M).m_pitch
                 o["with_both_skips"] = {"ms_per_step": rd["ms_per_step"], "cells_per_s": rd["cells_per_s"], "launch_ms": rd["layer_loop_ms"],
-                                        "hbm_frac": 2 * 4 * wk.B * wk.Lmax * wk.S * pitch4 / (rd["layer_loop_ms"] * 1e-3) / (hbm_gbs * 1e9),
+                                        "hbm_frac": 2 * 4 * int(np.sum(wk.L)) * wk.S * pitch4 / (rd["layer_loop_ms"] * 1e-3) / (hbm_gbs * 1e9),
                                         "opt_cost_sum": rd["opt_cost_sum"], "opt_cost_sum_plain": rk["opt_cost_sum"]}
                 del sbd
             # the same step replayed from a CUDA graph (launch latency matters for the small workloads)

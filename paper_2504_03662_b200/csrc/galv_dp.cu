@@ -436,7 +436,12 @@ constexpr int kDescRing = 16;
 // the result is min(low half, high half) + the column's base.  Exact: only differences are formed, nothing
 // is rounded, clamped candidates stay above every possible winner.  The whole tile (all S rows) comes from
 // the table as int32 into ONE buffer and is rebased by the consumer warps into one of two packed stages, so
-// the next tile's load runs under this tile's inner loop.
+// the next tile's load runs under this tile's inner loop.  Warps NC+4.. are further store warps there.
+//
+// Dominated rows left out (DOM, opt-in): the same bound says that a previous-layer row clamped in every column
+// of a warp group's 128-column tile contributes nothing to that tile.  The packed variant notes the live row
+// pairs while it rebases; the 32-bit variant (all S <= 64 rows in one stage) scans its columns first.  Either
+// way the group ORs its live rows together, meets at a barrier and relaxes only those.  Same results.
 template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false, bool DOM = false>
 __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
