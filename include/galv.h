@@ -75,9 +75,9 @@ extern "C" {
 #define GALV_SKIP_DOMINATED 8192 /* a candidate more than the largest transition entry above its column's best
                                     previous-layer value cannot win or tie; rows (row pairs in the packed loop) that
                                     are such in all 128 columns of a warp group's tile are left out of the inner
-                                    loop.  Same tables; the work then depends on the spread of the costs.  Honoured
-                                    by the one-launch kernels without argmin table when S <= 64 (and, in the 32-bit
-                                    loop, a tile's S rows fit one stage); ignored elsewhere. */
+                                    loop.  Same tables (argmin table included); the work then depends on the spread
+                                    of the costs.  Honoured when S <= 64 and, in the 32-bit loop, a tile's S rows fit
+                                    one stage; ignored elsewhere (GALV_KERNEL_REFERENCE among them). */
 
 typedef struct galv_ctx galv_ctx;
 

@@ -1251,7 +1251,14 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
 #pragma unroll
                             for (int j = 0; j < TM; ++j)
 #pragma unroll
-                                for (int u = 0; u < TS; ++u) acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                                for (int u = 0; u < TS; ++u) {
+                                    if (ARG) {                  // rows come in ascending order: the lowest row wins a tie
+                                        const int cand = c[j] + t[u];
+                                        if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = r; }
+                                    } else {
+                                        acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                                    }
+                                }
                         }
                     }
                 }
@@ -1398,12 +1405,14 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
                        bool packed)
 {
     auto kern = layer_tiled_kernel<TM, NSG, NMS, ARG, false>;
+    auto kern_dom = layer_tiled_kernel<TM, NSG, NMS, ARG, false, false, true>;
     auto kern_multi = layer_tiled_kernel<TM, NSG, NMS, false, true>;
     auto kern_packed = layer_tiled_kernel<TM, NSG, NMS, false, true, true>;
     auto kern_packed_dom = layer_tiled_kernel<TM, NSG, NMS, false, true, true, true>;
     auto kern_multi_dom = layer_tiled_kernel<TM, NSG, NMS, false, true, false, true>;
     if (!maps) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kern_dom, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_multi, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed_dom, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
@@ -1421,7 +1430,10 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
         const bool dom = a.skip_dom && pl.nkc == 1 && a.S <= 64;
         return cudaLaunchCooperativeKernel(dom ? (const void*)kern_multi_dom : (const void*)kern_multi, dim3(pl.grid), dim3((NSG * NMS + 4) * 32), args, (size_t)pl.smem, st);
     }
-    kern<<<pl.grid, (NSG * NMS + 4) * 32, pl.smem, st>>>(a, pl, l_first, l_last, maps[0], maps[1]);
+    if (a.skip_dom && pl.nkc == 1 && a.S <= 64)
+        kern_dom<<<pl.grid, (NSG * NMS + 4) * 32, pl.smem, st>>>(a, pl, l_first, l_last, maps[0], maps[1]);
+    else
+        kern<<<pl.grid, (NSG * NMS + 4) * 32, pl.smem, st>>>(a, pl, l_first, l_last, maps[0], maps[1]);
     return cudaGetLastError();
 }
 

@@ -544,19 +544,26 @@ def test_dominated_rows_left_out(orc, galv, S, M, trans_hi, time_hi):
     w.mem_q[3, 0, :] = M // 2                                    # the lower half of every later column is +inf
     for flags in (gb.STORE_C_FULL | gb.SKIP_DOMINATED, gb.SKIP_DOMINATED, gb.STORE_C_FULL | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE,
                   gb.STORE_C_FULL | gb.SKIP_DOMINATED | gb.KERNEL_NO_PACKED,            # the 32-bit loop's variant
-                  gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE | gb.KERNEL_NO_PACKED):
+                  gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE | gb.KERNEL_NO_PACKED,
+                  gb.STORE_C_FULL | gb.STORE_ARGMIN | gb.SKIP_DOMINATED,                # one launch per layer, argmin table
+                  gb.STORE_ARGMIN | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE,
+                  gb.STORE_C_FULL | gb.KERNEL_PER_LAYER | gb.SKIP_DOMINATED):
         sb = SearchBuffers(galv, w, flags)
         sb.dp_search(); sb.backtrack()
-        packable = S % 4 == 0 and int(w.trans_q.max()) <= 32767 and not flags & gb.KERNEL_NO_PACKED
+        packable = (S % 4 == 0 and int(w.trans_q.max()) <= 32767
+                    and not flags & (gb.KERNEL_NO_PACKED | gb.STORE_ARGMIN | gb.KERNEL_PER_LAYER))
         assert galv.galv_dp_search_path(sb.shape, sb.workspace) == packable
         res = sb.results()
         for i in range(B):
             Li = int(w.L[i])
             r = orc.search(w.time_q[i, :Li], w.mem_q[i, :Li], w.trans_q[i], M)
             assert res["status"][i] == r["status"] and res["opt_cost"][i] == r["opt_cost"], (flags, i)
-            if flags & gb.STORE_C_FULL:
+            if flags & (gb.STORE_C_FULL | gb.STORE_ARGMIN):
                 assert (res["plan"][i, :Li] == r["plan"]).all(), (flags, i)
+            if flags & gb.STORE_C_FULL:
                 assert (sb.table(i)[:Li] == r["C"]).all(), (flags, i)
+            if flags & gb.STORE_ARGMIN:
+                assert (sb.argmin_table(i)[:Li] == r["A"]).all(), (flags, i)
 
 
 def test_packed_path_with_costs_near_the_limit(orc, galv):
