@@ -381,6 +381,10 @@ def main():
                              "searches_per_s": rd["searches_per_s"], "opt_cost_sum": rd["opt_cost_sum"],
                              "launch_ms": rd["layer_loop_ms"],
                              "hbm_frac": hbm_bytes / (rd["layer_loop_ms"] * 1e-3) / (hbm_gbs * 1e9),
+                             "roofline": {"bound": "hbm", "achieved": hbm_bytes / (rd["layer_loop_ms"] * 1e-3) / 1e9, "peak": hbm_gbs,
+                                          "unit": "GB/s", "frac": hbm_bytes / (rd["layer_loop_ms"] * 1e-3) / (hbm_gbs * 1e9),
+                                          "traffic": None, "peak_source": "of measured" if peaks else "of fallback",
+                                          "algorithmic_bytes_per_launch": hbm_bytes},
                              "note": "part of the relaxations is proved unnecessary and left out: no ALU-roofline fraction"}
                 del sbd
                 torch.cuda.empty_cache()
