@@ -1150,6 +1150,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
             if (lane == 0) mbar_arrive(&out_full);            // release: the staging writes come before it
         }
     }
+    const int kmax = (DOM && !P16) ? a.maxmem[1] : 0;      // largest transition entry (read once: a global load inside the loop waits behind the SM's stores)
     for (int it = 0;; ++it) {
         int l = 0, mw = 0, nj = 0;
         ItemPos pos = {0, 0, 0};
@@ -1203,7 +1204,6 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                 uint32_t* const live_w = reinterpret_cast<uint32_t*>(meta0 + st * META + 2 * SB + 4 + 2 * ms);
                 if (kn > 0) {
                     constexpr int CW = (32 * TM + NSG - 1) / NSG;   // columns of the group each of its warps scans
-                    const int kmax = a.maxmem[1];
                     const int cend = min(sg * CW + CW, 32 * TM);
                     uint32_t lo = 0, hi = 0;
                     for (int c0 = sg * CW; c0 < cend; c0 += 32) {
