@@ -438,6 +438,18 @@ def main():
             del sbk, g
             torch.cuda.empty_cache()
         line["others"] = others
+        # The argmin-table mode (one launch per layer, at least three ALU operations per relaxation), plain and
+        # with dominated rows left out: whole steps on config 4 and on the first 40 layers of config 3
+        # (its full argmin + cost tables would not leave room for the other buffers of this run).
+        amode = {}
+        for wk in (workload_for(3, 0, 0, 40), workload_for(4)):
+            for key, fl in (("plain", 0), ("dominated_rows_skipped", gb.SKIP_DOMINATED)):
+                sba, ra = bench_workload(torch, galv, wk, 5, 3, barrier, flags=gb.STORE_ARGMIN | fl)
+                amode.setdefault(wk.name, {})[key] = {"ms_per_step": ra["ms_per_step"], "layer_loop_ms": ra["layer_loop_ms"],
+                                                      "cells_per_s": ra["cells_per_s"], "opt_cost_sum": ra["opt_cost_sum"]}
+                del sba
+                torch.cuda.empty_cache()
+        line["argmin_table_mode"] = amode
         line["cost_model_scaled"] = cost_model_scaled(torch, galv, hbm_gbs, barrier)
 
     if rank == 0 and world == 1 and not args.no_cpu:
