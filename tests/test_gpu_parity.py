@@ -372,6 +372,49 @@ def test_one_launch_against_reference_kernel_on_many_shapes(galv, block):
         torch.cuda.empty_cache()
 
 
+@pytest.mark.skipif(not os.environ.get("GALV_SOAK"), reason="long random-shape soak: set GALV_SOAK=<blocks of 10 shapes>")
+def test_soak_random_shapes_and_flags(galv):
+    """The stress above on many more shapes, with every kernel-selecting flag drawn at random (packed / 32-bit loop,
+    per layer, argmin table, both skipping flags): tables, optima and plans against the one-thread-per-cell kernel."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    choices = [0, gb.SKIP_INFEASIBLE, gb.SKIP_DOMINATED, gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE, gb.KERNEL_NO_PACKED,
+               gb.KERNEL_NO_PACKED | gb.SKIP_DOMINATED, gb.STORE_ARGMIN, gb.STORE_ARGMIN | gb.SKIP_DOMINATED,
+               gb.KERNEL_PER_LAYER | gb.SKIP_DOMINATED]
+    for block in range(int(os.environ["GALV_SOAK"])):
+        rng = np.random.default_rng(77000 + block)
+        for case in range(10):
+            S = int(rng.choice([1, 4, 5, 8, 12, 24, 31, 32, 36, 48, 60, 64, 65, 100, 130, 256]))
+            Lmax = int(rng.integers(2, 40))
+            M = int(rng.integers(10, 6000))
+            pitch = (M + 32) // 32 * 32
+            B = int(max(1, min(rng.integers(1, 200), 3.0e8 // (Lmax * S * pitch * 4))))
+            mem_hi = int(rng.choice([3, M // 20 + 3, M // 3 + 3, 2 * M + 3]))
+            w = inputs.random_tables(900000 + 100 * block + case, B, Lmax, S, M, ragged=bool(rng.integers(0, 2)),
+                                     mem_lo=int(rng.integers(0, 3)), mem_hi=mem_hi,
+                                     trans_hi=int(rng.choice([0, 7, 50, 3000, 32767, 32768, 50000])),
+                                     time_hi=int(rng.choice([10, 1000, 10 ** 5, 3 * 10 ** 6])))
+            if rng.integers(0, 3) == 0:
+                w.mem_q[:, int(rng.integers(0, Lmax)), :] += M // 2
+            ref = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_REFERENCE)
+            ref.dp_search(); ref.backtrack()
+            one = SearchBuffers(galv, w, gb.STORE_C_FULL | int(rng.choice(choices)))
+            for _ in range(2):
+                one.C.fill_(-7)
+                one.dp_search(); one.backtrack()
+                torch.cuda.synchronize()
+                st = ref.status.cpu().numpy()
+                assert (one.status.cpu().numpy() == st).all(), (block, case)
+                assert torch.equal(one.opt_cost, ref.opt_cost) and torch.equal(one.plan, ref.plan), (block, case)
+                for i in np.flatnonzero(st == 0):
+                    Li = int(w.L[i])
+                    assert torch.equal(one.C[i, :Li], ref.C[i, :Li]), (block, case, int(i), S, Lmax, M, B)
+                assert torch.equal(one.C_last[st == 0], ref.C_last[st == 0]), (block, case)
+            del ref, one
+            torch.cuda.empty_cache()
+
+
 def test_kernel_span_statistics(galv):
     """The timing hook keeps one event pair per profiled search and reports mean, shortest, longest."""
     import torch
