@@ -36,7 +36,9 @@
  * Cost model: FLOP count, x3/x4 factor, ring all-reduce byte counts and unit
  * conversion are pinned by closed forms; the memory-state, activation,
  * ZeRO-3 traffic, sequence-parallel and transition formulas are this build's
- * own accounting and are "parity unpinned" beyond self-consistency checks.
+ * own accounting (the paper gives none): the code is pinned to the stated
+ * formulas by hand-worked values, the formulas themselves have no outside
+ * truth and are "parity unpinned" in that sense.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -355,10 +357,13 @@ void orc_prune(int B, int Lmax, int S, const int32_t *L, const int32_t *time, co
  * stage made of layers a .. a+n-1 (ORC_INF when nothing fits); a pipeline runs at the pace of its
  * slowest stage, so the cut minimises the largest stage optimum:
  *   f[1][b] = opt(0,b),   f[k][b] = min_{k-1 <= a < b} max( f[k-1][a], opt(a,b) ).
- * cuts[0] = 0 < cuts[1] < ... < cuts[P] = Lm.  Several cuts can share the optimal bottleneck; the
- * one reported is the one the recurrence defines: walking back from the end, the lowest a attaining
- * f[k][b] is taken, so every prefix of the partition is itself cut optimally (not merely below the
- * bottleneck).  bottleneck = ORC_INF and cuts = -1 when no partition is feasible or P > Lm.
+ * cuts[0] = 0 < cuts[1] < ... < cuts[P] = Lm.  Several cut sets can share the optimal bottleneck.
+ * The one reported, stated without the recurrence: among the cut sets whose every prefix (the first
+ * k stages, k = 1..P) has the smallest bottleneck that any k-stage cut of the same layers can have,
+ * the one smallest in the order (cuts[P-1], cuts[P-2], ..., cuts[1]).  The walk back from the end
+ * that takes the lowest a attaining f[k][b] yields exactly that set (the tests enumerate all cut
+ * sets on tie-heavy models and compare the cuts themselves).
+ * bottleneck = ORC_INF and cuts = -1 when no partition is feasible or P > Lm.
  */
 void orc_stage_partition(int Lm, int P, const int32_t *range_opt, int32_t *cuts, int32_t *bottleneck)
 {

@@ -74,6 +74,16 @@ def test_config3_unjittered_values(orc):
     assert (tq[0, 63], mq[0, 63]) == (189635, 33) and (tq[1, 63], mq[1, 63]) == (272098, 65)
     assert (tq[0, 37], mq[0, 37]) == (280724, 127) and (tq[1, 37], mq[1, 37]) == (434245, 91)
     assert 80 * (33 + 65) <= w.M                         # the cheapest plan just fits
+    # Resharding entries that toggle sequence parallelism, worked by hand (activation = seq*h*2 B = 67 108 864 B,
+    # 450 GB/s, 10 ns units; factor = (k-1)/k for the tp change + (tp_dst-1)/tp_dst for the toggle):
+    #   tp8/sp0 -> tp8/sp1: 7/8      -> 13 048.9 ;  tp2/sp0 -> tp4/sp1: 1/2 + 3/4 -> 18 641.4
+    #   tp4/sp1 -> tp2/sp0: 1/2 + 1/2 -> 14 913.1 ;  tp1/sp0 -> tp8/sp1: 7/8 + 7/8 -> 26 097.9
+    st = w.strat
+    idx = lambda tp, sp: int(np.flatnonzero((st["tp"] == tp) & (st["sp"] == sp) & (st["zero"] == 0) & (st["ckpt"] == 0))[0])
+    assert (idx(8, 0), idx(8, 1), idx(2, 0), idx(4, 1), idx(1, 0)) == (48, 49, 16, 33, 0)
+    assert xq[48, 49] == 13049 and xq[16, 33] == 18641 and xq[33, 16] == 14913 and xq[0, 49] == 26098
+    assert xq[49, 48] == 13049                           # same destination tp: the toggle costs the same both ways
+    assert xq[0, 1] == 0                                 # toggling at tp = 1 moves nothing
     # jitter stays within +-20 %
     wj = inputs.config3()
     assert (wj.inst["flops_rate"] >= 0.8e15).all() and (wj.inst["flops_rate"] < 1.2e15).all()

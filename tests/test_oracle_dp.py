@@ -72,6 +72,35 @@ def test_tie_order_is_last_layer_first(orc):
     assert numpy_enumerate(time, mem, trans, 0) == (10, [1, 0])
 
 
+def test_config0_values_printed_in_the_build_brief(orc):
+    """Config 0 under the stated generator, against figures the build brief prints for it (computed there by
+    an independent throw-away enumeration, not by this oracle): first generator rows, optimum / plan / memory
+    at four budgets, two table rows with their argmins, the count of finite cells and their sum.  A different
+    draw order, a transposed trans matrix or a shifted budget index changes at least one of them."""
+    w = inputs.config0()
+    t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
+    assert t[0].tolist() == [9921, 1805, 4023, 6050, 2684, 4956]
+    assert m[0].tolist() == [10, 12, 9, 17, 23, 11]
+    assert x[0].tolist() == [0, 1321, 1646, 1918, 1077, 747]
+    Ct, At = orc.dp(t, m, x, w.M)
+    assert Ct[3][64].tolist() == [12694, 12368, 9749, 7693, 11027, 10728]
+    assert At[3][64].tolist() == [4, 4, 4, 4, 4, 4]
+    assert Ct[1][20].tolist() == [5331, 2881, 7529, 14392, 12411, INF]
+    assert At[1][20].tolist() == [1, 1, 1, 2, 1, 255]
+    finite = Ct < INF
+    assert Ct.size == 1560 and int(finite.sum()) == 1069 and int(Ct[finite].astype(np.int64).sum()) == 8891677
+    for budget, want in ((64, (7693, [1, 1, 4, 3], 45)), (40, (7803, [1, 1, 3, 3], 36)),
+                         (30, (10341, [1, 1, 3, 2], 29)), (20, (16861, [2, 2, 5, 2], 18))):
+        for A in (None, At):
+            opt, plan, used, st = orc.backtrack(t, m, x, Ct, A, budget)
+            assert (opt, plan.tolist(), used, st) == (want[0], want[1], want[2], 0), budget
+        assert orc.brute_force(t, m, x, budget)[:3][0] == want[0]
+    for budget in (0, 9, 17):
+        assert orc.backtrack(t, m, x, Ct, None, budget)[0] == INF
+    assert orc.backtrack(t, m, x, Ct, None, 18)[0] < INF
+    assert orc.brute_force(t, m, x, 64)[3] == 1231          # feasible plans of the 1296
+
+
 def test_config0_against_exhaustive_golden(orc):
     w = inputs.config0()
     t, m, x = w.time_q[0], w.mem_q[0], w.trans_q[0]
