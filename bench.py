@@ -44,7 +44,17 @@ NCU_TRAFFIC_BYTES_PER_LAYER = {"config3_heterogeneous": 532.7e6, "config4_resear
 
 
 def workload_for(k: int, rank: int = 0, batch: int = 0, layers: int = 0):
-    w = inputs.CONFIGS[k]()
+    """Workload k; ranks > 0 of a multi-GPU run get other instances of the same shape (other seed / other jitter)."""
+    if rank and k in (0, 4):
+        w = inputs.CONFIGS[k](seed=(0 if k == 0 else 7) + 1000 * rank)
+    else:
+        w = inputs.CONFIGS[k]()
+    if rank and w.has_model:
+        # the same model searched under other measured rates: two draws per instance scale the FLOP rate and the
+        # link bandwidth by a factor in [0.8, 1.2), as the heterogeneous workload does on rank 0
+        u = inputs._unit(inputs.splitmix64(3 + 1000 * rank, 2 * w.B)).reshape(w.B, 2)
+        w.inst["flops_rate"] = 1e15 * (0.8 + 0.4 * u[:, 0])
+        w.inst["bw_tp"] = w.inst["bw_dp"] = 450e9 * (0.8 + 0.4 * u[:, 1])
     if batch or layers:
         # trimmed copy of the workload (first `batch` instances, first `layers` layers) for profiler captures
         w = w.take(slice(0, batch or w.B))
@@ -56,12 +66,25 @@ def workload_for(k: int, rank: int = 0, batch: int = 0, layers: int = 0):
             else:
                 w.time_q = np.ascontiguousarray(w.time_q[:, :layers]); w.mem_q = np.ascontiguousarray(w.mem_q[:, :layers])
         w.name += f"[B={w.B},L={w.Lmax}]"
-    if rank and w.has_model and k == 3:
-        # other ranks search other jittered instances of the same shape
-        u = inputs._unit(inputs.splitmix64(3 + 1000 * rank, 2 * w.B)).reshape(w.B, 2)
-        w.inst["flops_rate"] = 1e15 * (0.8 + 0.4 * u[:, 0])
-        w.inst["bw_tp"] = w.inst["bw_dp"] = 450e9 * (0.8 + 0.4 * u[:, 1])
     return w
+
+
+def input_checksums(w) -> dict:
+    """FNV-1a-64 of the first 64 KiB of every input array of the workload (hex)."""
+    arrays = (("L", w.L), ("layers", w.layers), ("strat", w.strat), ("inst", w.inst),
+              ("time_q", w.time_q), ("mem_q", w.mem_q), ("trans_q", w.trans_q))
+    return {name: f"{inputs.fnv1a64(a):016x}" for name, a in arrays if a is not None}
+
+
+def spawn_ranks(n: int) -> int:
+    """Re-run this command as n ranks of one node (one process per GPU, NCCL rendezvous on the loopback address)."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 # ------------------------------------------------------------------ CPU oracle legs
@@ -254,6 +277,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "galv" else args.warmup
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))            # no launcher around this process: start the ranks here
 
     import torch
     import torch.distributed as dist
@@ -265,9 +290,16 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the search has no CPU path")
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if torch.cuda.device_count() < world:
+        raise SystemExit(f"bench.py: {world} ranks but only {torch.cuda.device_count()} CUDA device(s) are visible")
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if rank == 0:
+            print(f"[bench] communicator: backend nccl {'.'.join(map(str, torch.cuda.nccl.version()))}, {world} ranks on one node, "
+                  f"used for the barrier and the max over ranks only (no collective on the data path)", file=sys.stderr)
 
     def barrier():
         if world > 1:
@@ -340,12 +372,28 @@ def main():
                                     + (" (two relaxations each in the packed 16-bit form)" if r["packed"] else "")},
     }
 
+    line["inputs_fnv1a64"] = input_checksums(w)
+    line["kernel_variant"] = line["roofline"]["kernel"]
     if rank == 0:
+        # The ALU peak measured on this GPU, in the run itself, by register-only probes of the very instruction the
+        # inner loop issues (relaxations per second: the packed instruction counts as the two it performs).
+        rf = line["roofline"]
+        rf["peak_derived"] = rf["peak"]
         try:
-            line["roofline"]["probe_gops"] = {k: galv.galv_probe_int_alu(i, 4096) / 1e9
-                                              for i, k in enumerate(("fused_addmin", "add_then_min", "add_xor_2ops"))}
+            fused = galv.galv_probe_int_alu(0, 4096) / 1e9
+            packed = galv.galv_probe_int_alu(3, 4096) / 1e9
+            rf["peak_measured"] = packed if r["packed"] else fused
+            rf["frac_of_measured"] = achieved / rf["peak_measured"]
+            rf["probe_fused_addmin_gops"] = fused
+            rf["probe_packed_addmin_u16x2_gops"] = packed
+            rf["probe_add_then_min_gops"] = galv.galv_probe_int_alu(1, 4096) / 1e9
+            rf["probe_add_xor_2ops_gops"] = galv.galv_probe_int_alu(2, 4096) / 1e9
+            rf["probe_min3_gops"] = galv.galv_probe_int_alu(4, 4096) / 1e9
+            rf["peak_measured_source"] = ("galv_probe_int_alu kind 3 (__viaddmin_u16x2, two relaxations per instruction)" if r["packed"]
+                                          else "galv_probe_int_alu kind 0 (__viaddmin_s32)")
         except gb.GalvError as e:      # diagnostic only
-            line["roofline"]["probe_gops"] = str(e)
+            rf["peak_measured"] = None
+            rf["probe_error"] = str(e)
         # HBM side of the roofline: every table cell written once and read once by the next layer
         from paper_2504_03662_b200.binding import make_shape
         pitch = make_shape(w.B, w.Lmax, w.S, w.M).m_pitch

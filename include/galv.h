@@ -140,7 +140,9 @@ size_t galv_dp_workspace_bytes(const galv_ctx* ctx, const galv_shape* shape);
  *   C[0][m][s] = time(0,s)                      if mem(0,s) <= m, else GALV_INF
  *   C[l][m][s] = time(l,s) + min_{s'} ( C[l-1][m-mem(l,s)][s'] + trans(s',s) )
  * GALV_INF where m < mem(l,s) or every candidate is GALV_INF.  A[l][m][s] is the
- * lowest minimising s' (255 for GALV_INF cells and on layer 0).
+ * lowest minimising s' (255 for GALV_INF cells and on layer 0; with S = 256 the
+ * value 255 is also a strategy index: read A only where C is finite, as
+ * galv_backtrack does).
  *
  * Before the recurrence every instance is validated: entries >= 0, L[i] in
  * 1..Lmax, and sum_l max_s time + (L-1)*max trans < GALV_INF.  status[i] is set
@@ -189,12 +191,21 @@ int galv_dp_search_path(galv_ctx* ctx, const galv_shape* shape, const void* work
  *
  * Arguments, results and status bits are those of galv_dp_search.  Shapes whose
  * galv_dp_workspace_bytes exceeds GALV_STATIC_WORKSPACE_BYTES are refused with
- * GALV_ERR_WORKSPACE (in practice: any batch that keeps the full table fits;
- * the rolling two-layer mode fits only small B*S*m_pitch).  The call itself
- * allocates nothing, on the host or the device.
+ * GALV_ERR_WORKSPACE.  What the scratch holds: a few int32 per instance and per
+ * layer; 4 bytes per (instance, layer) and per (instance, tile of 128 budget
+ * columns); B*S*S*2 bytes of packed transition rows when the packed 16-bit
+ * loop may run (S <= 64, S % 4 == 0, neither GALV_KERNEL_NO_PACKED nor
+ * GALV_STORE_ARGMIN nor GALV_KERNEL_PER_LAYER; times Lmax with
+ * GALV_TRANS_PER_LAYER); and 2*B*S*m_pitch*4 bytes when the full table is not
+ * kept.  So batches of a few hundred instances with the full table fit; large
+ * batches fit only with GALV_KERNEL_NO_PACKED (B = 1024, S = 32 needs 2 MiB
+ * for the packed rows alone), and the rolling two-layer mode only for small
+ * B*S*m_pitch.  Ask galv_dp_workspace_bytes.  The call itself allocates
+ * nothing, on the host or the device.
  *
- * The first call on a device looks up the array's device address (once per
- * device); make that first call outside any stream capture.  All calls share
+ * The first call on a device looks up the array's device address and, like the
+ * first launch of any kernel, makes the CUDA runtime load the library's device
+ * code (once per device); make that first call outside any stream capture.  All calls share
  * the one array: what has to start from zero is cleared by each call, and two
  * calls that overlap on the GPU (different streams, or different contexts on
  * the same device) race on it — serialise them.
@@ -359,7 +370,10 @@ int galv_search_host(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
  * per second in *ops_per_s (host pointer).  kind 0: fused add-then-min, counted
  * as one operation per min-plus relaxation; kind 1: add then min written as two
  * C statements (however the compiler lowers them), counted per relaxation;
- * kind 2: add then xor, two plain int32 operations, both counted.  Synchronises.
+ * kind 2: add then xor, two plain int32 operations, both counted; kind 3: the
+ * packed add-then-min on two unsigned 16-bit halves (the instruction of the
+ * packed 16-bit inner loop), counted as the two relaxations it performs;
+ * kind 4: three-input minimum, counted per instruction.  Synchronises.
  */
 int galv_probe_int_alu(galv_ctx* ctx, int kind, int iters, double* ops_per_s, void* stream);
 

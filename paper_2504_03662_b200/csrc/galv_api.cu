@@ -369,7 +369,7 @@ int galv_layer_loop_ms_stats(galv_ctx* ctx, float* mean_ms, float* min_ms, float
 
 int galv_probe_int_alu(galv_ctx* ctx, int kind, int iters, double* ops_per_s, void* stream)
 {
-    if (!ctx || !ops_per_s || iters < 1 || kind < 0 || kind > 2) return GALV_ERR_INVALID_ARG;
+    if (!ctx || !ops_per_s || iters < 1 || kind < 0 || kind > 4) return GALV_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     cudaEvent_t e0, e1;
     cudaError_t e;

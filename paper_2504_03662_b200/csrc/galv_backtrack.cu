@@ -39,7 +39,8 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, lon
         for (int l = lane; l < Lmax; l += 32) pl[l] = -1;
     __syncwarp();          // lane 0 overwrites entries other lanes have just cleared
     const int bud = budget ? budget[i] : M;
-    const bool skip = (st0 & (GALV_STATUS_BAD_INPUT | GALV_STATUS_OVERFLOW_RISK)) != 0 || bud < 0 || bud > M;
+    // a search whose bounded waits ran out left void tables: not walked either
+    const bool skip = (st0 & (GALV_STATUS_BAD_INPUT | GALV_STATUS_OVERFLOW_RISK | GALV_STATUS_TIMEOUT)) != 0 || bud < 0 || bud > M;
     if (skip) {
         if (lane == 0) {
             opt_cost[i] = kInf;
@@ -98,6 +99,10 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, lon
         const int mm = __shfl_sync(0xffffffffu, msel, s & 31);
         const int tt = __shfl_sync(0xffffffffu, tsel, s & 31);
         used += mm;
+        if (mm > m) {                  // cannot happen on consistent tables: the cell would be +inf; never index below column 0
+            if (lane == 0) status[i] = st0 | GALV_STATUS_BAD_INPUT;
+            break;
+        }
         if (l == 0) break;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {                          // rows of layer l-1, needed one step from now

@@ -18,8 +18,9 @@
 // A layer needs the previous one.  With the full table kept, all layers run in one
 // cooperative launch: CTAs publish finished tiles in global counters and start a
 // tile of the next layer as soon as the tiles it reads are published (bounded
-// waits).  With an argmin table or the two-layer rolling buffer: one launch per
-// layer.  Either way plain stream work, capturable in a CUDA graph.
+// waits); on the two-layer rolling buffer a tile also waits for the readers of the
+// cells it overwrites.  With an argmin table: one launch per layer.  Either way plain
+// stream work, capturable in a CUDA graph.
 
 #include <cuda.h>
 
@@ -173,7 +174,7 @@ __global__ void validate_kernel(int B, int Lmax, int S, int M, long long tl, con
     }
     const int32_t* x = trans_q + (size_t)i * (tl ? (size_t)Lmax * S * S : (size_t)S * S);
     const int xl0 = tl ? 1 : 0, xl1 = tl ? Li : 1;            // matrices in use
-    for (int k = threadIdx.x; k < (xl1 - xl0) * S * S; k += blockDim.x) {
+    for (long long k = threadIdx.x; k < (long long)(xl1 - xl0) * S * S; k += blockDim.x) {
         const int v = x[(size_t)xl0 * S * S + k];
         bad |= (v < 0);
         tmax = max(tmax, v);
@@ -1480,7 +1481,7 @@ WsLayout galv_ws_layout(const galv_shape* sh)
     w.front = off;    off = align256(off + (size_t)sh->B * sh->Lmax * 4);
     w.tile_done = off; off = align256(off + (size_t)sh->B * ((sh->M + 128) / 128) * 4);   // per (instance, tile of >= 128 columns)
     w.trans_p = off;                                           // packed trans rows for the 16-bit path (S <= 64, S % 4 == 0)
-    if (sh->S <= 64 && sh->S % 4 == 0)
+    if (sh->S <= 64 && sh->S % 4 == 0 && !(sh->flags & (GALV_KERNEL_NO_PACKED | GALV_STORE_ARGMIN | GALV_KERNEL_PER_LAYER | GALV_KERNEL_REFERENCE)))
         off = align256(off + (size_t)sh->B * ((sh->flags & GALV_TRANS_PER_LAYER) ? sh->Lmax : 1) * (sh->S / 2) * sh->S * 4);
     w.roll = off;
     if (!(sh->flags & GALV_STORE_C_FULL)) off = align256(off + (size_t)2 * sh->B * sh->S * sh->m_pitch * 4);
@@ -1602,7 +1603,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
                                        (sh->flags & GALV_SKIP_INFEASIBLE) ? a.front : nullptr);
     schedule_kernel<<<1, 1024, 0, st>>>(B, Lmax, a.M, pl.tmb, pl.ntiles_m, pl.nsb, a.L, a.status, a.order, a.nactive, a.scratch,
                                          a.minmem_l, a.ntiles, a.istart, a.tcount, will_p16, a.err + 1);
-    {
+    auto base_layer = [&]() {
         int gx = (a.m_pitch + 255) / 256;
         if (gx > 8) gx = 8;
         for (int b0 = 0; b0 < B; b0 += 65535) {           // grid.z limit
@@ -1616,7 +1617,8 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
             s.roll += (size_t)b0 * S * a.m_pitch;
             base_layer_kernel<<<dim3(gx, S, nb), 256, 0, st>>>(s);
         }
-    }
+    };
+    base_layer();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
     CUtensorMap maps[4];
@@ -1656,9 +1658,15 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
         e = will_p16 ? launch_tiled<false>(ap, pl, 1, Lmax, st, maps, true) : cudaSuccess;
         if (e == cudaSuccess) e = launch_tiled<false>(ap, pl, 1, Lmax, st, maps);
         if (e == cudaErrorCooperativeLaunchTooLarge) {
-            // the grid cannot be co-resident right now (SMs taken by another context): one launch per layer instead
+            // the grid cannot be co-resident right now (SMs taken by another context): one launch per layer instead.
+            // If the packed kernel was accepted before the 32-bit one was refused it may have run every layer, and on
+            // the rolling buffer that overwrote layer 0: write the base layer again behind it.
             (void)cudaGetLastError();
             ap.tile_done = nullptr;
+            if (!a.C && will_p16) {
+                base_layer();
+                if ((e = cudaGetLastError()) != cudaSuccess) return e;
+            }
         } else if (e != cudaSuccess) {
             return e;
         } else {

@@ -26,7 +26,9 @@ __global__ void __launch_bounds__(256) probe_kernel(int iters, int seed)
                 int& a = acc[j * 8 + u];
                 if (KIND == 0) a = __viaddmin_s32(a, t[u], c[j]);          // one instruction per relaxation
                 else if (KIND == 1) { int v = a + t[u]; a = v < c[j] ? v : c[j]; }   // as the compiler lowers it
-                else a = (a + t[u]) ^ c[j];                                 // two plain integer operations
+                else if (KIND == 2) a = (a + t[u]) ^ c[j];                  // two plain integer operations
+                else if (KIND == 3) a = (int)__viaddmin_u16x2((unsigned)c[j], (unsigned)t[u], (unsigned)a);   // packed 16-bit pair: two relaxations
+                else a = __vimin3_s32(a, t[u], c[j]);                       // three-input minimum (side work of the packed loop)
             }
     }
     int r = 0;
@@ -42,8 +44,11 @@ cudaError_t galv_probe_launch(const galv_ctx* ctx, int kind, int iters, int32_t*
     const int blocks = ctx->num_sms * 8, threads = 256;
     if (kind == 0) probe_kernel<0><<<blocks, threads, 0, st>>>(iters, 12345);
     else if (kind == 1) probe_kernel<1><<<blocks, threads, 0, st>>>(iters, 12345);
-    else probe_kernel<2><<<blocks, threads, 0, st>>>(iters, 12345);
-    // kinds 0 and 1 count relaxations (add+min pairs); kind 2 counts both of its operations
-    *ops = (long long)blocks * threads * 32 * iters * (kind == 2 ? 2 : 1);
+    else if (kind == 2) probe_kernel<2><<<blocks, threads, 0, st>>>(iters, 12345);
+    else if (kind == 3) probe_kernel<3><<<blocks, threads, 0, st>>>(iters, 12345);
+    else probe_kernel<4><<<blocks, threads, 0, st>>>(iters, 12345);
+    // kinds 0 and 1 count relaxations (add+min pairs); kind 2 counts both of its operations; kind 3 counts the
+    // two relaxations each packed instruction performs; kind 4 counts instructions
+    *ops = (long long)blocks * threads * 32 * iters * ((kind == 2 || kind == 3) ? 2 : 1);
     return cudaGetLastError();
 }

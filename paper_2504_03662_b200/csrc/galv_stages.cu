@@ -25,7 +25,7 @@ __global__ void layer_optima_kernel(int B, int Lmax, int S, int M, int m_pitch, 
     const int i = (int)(w / Lmax), l = (int)(w - (long long)i * Lmax);
     int best = kInf;
     const int bud = budget ? budget[i] : M;
-    const bool ok = (status[i] & (GALV_STATUS_BAD_INPUT | GALV_STATUS_OVERFLOW_RISK)) == 0 && l < L[i] && bud >= 0 && bud <= M;
+    const bool ok = (status[i] & (GALV_STATUS_BAD_INPUT | GALV_STATUS_OVERFLOW_RISK | GALV_STATUS_TIMEOUT)) == 0 && l < L[i] && bud >= 0 && bud <= M;
     if (ok)
         for (int s = lane; s < S; s += 32) best = min(best, C[(((size_t)i * Lmax + l) * S + s) * m_pitch + bud]);
 #pragma unroll

@@ -117,13 +117,14 @@ class Workload:
 
 # --------------------------------------------------------------------------- random tables
 
-def config0() -> Workload:
+def config0(seed: int = 0) -> Workload:
     """Tiny search: uniform time in [100,10000], mem in [1,24], trans in [0,2000], zero diagonal.
 
-    Draw order: all time[l][s] (l-major), all mem[l][s], then trans row-major.
+    Draw order: all time[l][s] (l-major), all mem[l][s], then trans row-major.  The workload is seed 0;
+    other seeds give other instances of the same shape (further ranks of a multi-GPU run).
     """
     L, S, M = 4, 6, 64
-    x = splitmix64(0, 2 * L * S + S * S)
+    x = splitmix64(seed, 2 * L * S + S * S)
     time = _randint(x[:L * S], 100, 10000).reshape(1, L, S)
     mem = _randint(x[L * S:2 * L * S], 1, 24).reshape(1, L, S)
     trans = _randint(x[2 * L * S:], 0, 2000).reshape(1, S, S)
@@ -131,7 +132,7 @@ def config0() -> Workload:
     return Workload("config0_tiny", 1, L, S, M, np.full(1, L, np.int32), time, mem, trans)
 
 
-def config4(B: int = 1024) -> Workload:
+def config4(B: int = 1024, seed: int = 7) -> Workload:
     """Re-search stress: log-normal time (mu = ln 5e5 ns, sigma = 0.5), mem in [8,128], dense trans in [0,5e4].
 
     Instance-major stream; per instance: time (two draws per value, Box-Muller
@@ -139,7 +140,7 @@ def config4(B: int = 1024) -> Workload:
     """
     L, S, M = 48, 32, 2048
     per = 2 * L * S + L * S + S * S
-    x = splitmix64(7, B * per).reshape(B, per)
+    x = splitmix64(seed, B * per).reshape(B, per)
     xt = x[:, :2 * L * S].reshape(B, L * S, 2)
     u1 = ((xt[..., 0] >> np.uint64(11)).astype(np.float64) + 1.0) * 2.0 ** -53
     u2 = _unit(xt[..., 1])
@@ -264,7 +265,7 @@ CONFIGS = {0: config0, 1: config1, 2: config2, 3: config3, 4: config4}
 
 
 def fnv1a64(a: np.ndarray) -> int:
-    """FNV-1a 64-bit checksum of an array's bytes (input fingerprint printed by the bench)."""
+    """FNV-1a 64-bit checksum of the first 64 KiB of an array's bytes (input fingerprint printed by the bench)."""
     h = 0xCBF29CE484222325
     for byte in np.ascontiguousarray(a).view(np.uint8).ravel()[: 1 << 16].tolist():
         h = ((h ^ byte) * 0x100000001B3) & 0xFFFFFFFFFFFFFFFF

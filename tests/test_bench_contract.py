@@ -46,8 +46,32 @@ def test_gpu_arm_line():
     assert r["bound"] in ("alu", "hbm") and r["unit"] and r["peak"] > 0
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and 0.3 < r["frac"] < 1.1
     assert r["traffic"] is None or r["traffic"] > 0
+    # the denominator measured in the same run, as plain top-level numbers
+    assert r["peak_derived"] == r["peak"] and r["peak_measured"] > 0.5 * r["peak"]
+    assert abs(r["frac_of_measured"] - r["achieved"] / r["peak_measured"]) < 1e-9
+    assert set(d["inputs_fnv1a64"]) >= {"L", "layers", "strat", "inst"} and d["kernel_variant"]
     c = d["clocks"]
     assert c["sm_mhz"] > 0 and c["sm_max_mhz"] >= c["sm_mhz"] and isinstance(c["reasons"], list)
     e = d["e2e"]
     assert e["unit"] == d["unit"] and 0 < e["value"] <= d["value"] * 1.05
     assert e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
+
+
+def test_gpus_flag_must_match_the_launcher():
+    """--gpus N under a launcher that started another number of ranks is refused, not silently run at N = 1."""
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"], capture_output=True,
+                         text=True, timeout=300, cwd=ROOT, env=env)
+    assert out.returncode != 0 and not [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert "CUDA device" in out.stderr or "--gpus 2" in out.stderr
+
+
+def test_per_rank_inputs_differ_but_keep_the_shape():
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    import bench
+    for k in range(5):
+        a, b = bench.workload_for(k, 0), bench.workload_for(k, 1)
+        assert (a.B, a.Lmax, a.S, a.M) == (b.B, b.Lmax, b.S, b.M) and (a.L == b.L).all()
+        assert bench.input_checksums(a) != bench.input_checksums(b), k
+        assert bench.input_checksums(a) == bench.input_checksums(bench.workload_for(k, 0))

@@ -40,8 +40,11 @@ def test_host_side_answers_without_a_device(lib):
     assert sh.m_pitch == 2912
     small = lib.galv_dp_workspace_bytes(None, C.byref(sh))
     assert 0 < small < 1 << 20
-    roll = lib.galv_dp_workspace_bytes(None, C.byref(gb.make_shape(16, 24, 24, 2880, gb.STORE_ARGMIN)))
-    assert roll >= small + 2 * 16 * 24 * 2912 * 4
+    roll = lib.galv_dp_workspace_bytes(None, C.byref(gb.make_shape(16, 24, 24, 2880, 0)))
+    assert roll >= small + 2 * 16 * 24 * 2912 * 4                # two rolling layers on top
+    # flags that rule the packed 16-bit loop out drop its packed transition rows from the workspace
+    lean = lib.galv_dp_workspace_bytes(None, C.byref(gb.make_shape(16, 24, 24, 2880, gb.STORE_C_FULL | gb.KERNEL_NO_PACKED)))
+    assert small - lean >= 16 * 12 * 24 * 4
     assert lib.galv_dp_workspace_bytes(None, C.byref(gb.make_shape(16, 24, 0, 2880))) == 0
     assert lib.galv_search_host_arena_bytes(None, C.byref(sh), 1) > 16 * 24 * 24 * 2912 * 4
     # entry points refuse a missing context before touching the device

@@ -82,3 +82,50 @@ def test_two_ranks_gather_the_whole_batch():
         for k in ("opt_cost", "plan", "mem_used", "status"):
             assert np.array_equal(np.asarray(got[rank][k]), want[k]), (rank, k)
     assert want["status"][4] == 2
+
+
+def _cuda_worker(port, q):
+    import torch
+    import torch.distributed as dist
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    from paper_2504_03662_b200.sharding import search_sharded
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    torch.cuda.set_device(0)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        galv = gb.Galv(0)
+
+        def local(sub):
+            sb = SearchBuffers(galv, sub, gb.STORE_C_FULL)
+            sb.step()
+            return sb.results()
+
+        out = {}
+        for name, w in (("ragged", inputs.config2()), ("tables", inputs.config4(B=40))):
+            res = search_sharded(w, local, torch.device("cuda", 0))
+            whole = local(w)
+            out[name] = all(np.array_equal(res[k], whole[k]) for k in ("opt_cost", "plan", "mem_used", "status"))
+            out[name + "_feasible"] = int((res["status"] == 0).sum())
+        galv.close()
+        q.put(out)
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.gpu
+@pytest.mark.timeout(300)
+def test_cuda_path_through_the_sharded_search_over_nccl():
+    """The sharded search with the CUDA path as the per-slice search, one rank, NCCL as the gather's backend:
+    the gathered results equal those of the unsharded run (the only multi-GPU form one GPU can run)."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    p = ctx.Process(target=_cuda_worker, args=(port, q))
+    p.start()
+    got = q.get(timeout=280)
+    p.join(timeout=30)
+    assert p.exitcode == 0
+    assert got["ragged"] and got["tables"] and got["ragged_feasible"] > 0 and got["tables_feasible"] == 40
