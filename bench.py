@@ -231,7 +231,9 @@ def cost_model_scaled(torch, galv, hbm_gbs, barrier, copies=8192):
             "gb_per_s": nbytes / t / 1e9, "frac_of_hbm": nbytes / t / 1e9 / hbm_gbs}
 
 
-def launches_per_step(w) -> int:
+def launches_per_step(w, cluster: bool = False) -> int:
+    if cluster:                                   # cost + trans kernels, ONE cluster kernel for the whole search, backtrack
+        return (2 if w.has_model else 0) + 1 + 1
     # cost + trans kernels, validate + schedule + base layer, ONE cooperative launch over all layers,
     # copy-last + finalize, backtrack; where the shape allows the packed 16-bit path, the kernel that packs
     # the trans rows and the launch of the other inner-loop variant (it returns at once) come on top
@@ -240,6 +242,7 @@ def launches_per_step(w) -> int:
 
 
 def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):
+    from paper_2504_03662_b200 import binding as gb
     from paper_2504_03662_b200.search import SearchBuffers
     sb = SearchBuffers(galv, w, flags)
     for _ in range(warmup):
@@ -248,12 +251,13 @@ def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):
     t = time_steps(torch, sb.step, steps, 0, barrier)
     step_ms = sorted(LAST_STEP_MS)
     layer_ms, layer_min, layer_max, layer_n = galv.galv_layer_loop_ms_stats()   # mean over the timed searches (the last 64)
-    packed = galv.galv_dp_search_path(sb.shape, sb.workspace)                   # which inner loop ran
+    path = galv.galv_dp_search_path(sb.shape, sb.workspace)                     # which kernel ran
+    packed, cluster = path == gb.PATH_TILED_PACKED, path == gb.PATH_CLUSTER
     galv.galv_set_profiling(False)
     res = sb.results()
     out = {"seconds": t, "ms_per_step": t / steps * 1e3, "cells_per_s": w.cells * steps / t,
            "relax_per_s": w.relaxations * steps / t, "searches_per_s": w.B * steps / t,
-           "layer_kernel_ms_avg": layer_ms / max(1, w.Lmax - 1), "layer_loop_ms": layer_ms, "packed": packed,
+           "layer_kernel_ms_avg": layer_ms / max(1, w.Lmax - 1), "layer_loop_ms": layer_ms, "packed": packed, "cluster": cluster,
            "ms_median": statistics.median(step_ms), "ms_best": step_ms[0], "layer_loop_ms_min": layer_min, "layer_loop_ms_max": layer_max, "layer_loop_launches_timed": layer_n,
            "feasible": int((res["status"] == 0).sum()), "opt_cost_sum": int(res["opt_cost"][res["status"] == 0].sum())}
     return sb, out
@@ -270,6 +274,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiler captures)")
     ap.add_argument("--no-packed", action="store_true", help="keep the 32-bit inner loop where the packed 16-bit one would run")
+    ap.add_argument("--no-cluster", action="store_true", help="keep the tiled kernels where the small-batch cluster kernel would run")
+    ap.add_argument("--instance", type=int, default=-1, help="search only this instance of the workload (single re-search latency)")
     ap.add_argument("--skip-dominated", action="store_true", help="run with GALV_SKIP_DOMINATED (profiler captures; the roofline keys then do not apply)")
     ap.add_argument("--batch", type=int, default=0, help="trim the workload to its first instances (profiler captures)")
     ap.add_argument("--layers", type=int, default=0, help="trim the workload to its first layers (profiler captures)")
@@ -313,12 +319,18 @@ def main():
         return float(t.item())
 
     galv = gb.Galv(local)
+    for _ in range(8):                                           # bring the clocks up before short workloads are timed
+        galv.galv_probe_int_alu(0, 4096)
     w = workload_for(args.workload, rank, args.batch, args.layers)
+    if args.instance >= 0:
+        w = w.take([args.instance])
+        w.name += f"[instance {args.instance}]"
     uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", "")
 
     with ClockSampler(uuid) as clk:
         sb, r = bench_workload(torch, galv, w, args.steps, args.warmup, barrier,
-                               flags=1 | (gb.KERNEL_NO_PACKED if args.no_packed else 0) | (gb.SKIP_DOMINATED if args.skip_dominated else 0))
+                               flags=1 | (gb.KERNEL_NO_PACKED if args.no_packed else 0) | (gb.SKIP_DOMINATED if args.skip_dominated else 0)
+                                     | (gb.KERNEL_NO_CLUSTER if args.no_cluster else 0))
     t = max_over_ranks(r["seconds"])
     clocks = clk.summary()
     value = world * w.cells * args.steps / t
@@ -353,7 +365,7 @@ def main():
                    "tables": "full C kept (int32), plan re-derived along the path",
                    "l2": "tables far larger than L2 (no flush needed)", "parallelism": f"instances x{world}"},
         "searches_per_s": world * w.B * args.steps / t, "relaxations_per_s": world * w.relaxations * args.steps / t,
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(w) * args.steps,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(w, r["cluster"]) * args.steps,
         "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_GOPS * (2 if r["packed"] else 1), "unit": "G add-min/s",
                      "frac": achieved / (ALU_PEAK_GOPS * (2 if r["packed"] else 1)),
                      "frac_of_32bit_peak": achieved / ALU_PEAK_GOPS,
@@ -364,8 +376,9 @@ def main():
                      "traffic_unit": "bytes per launch (ncu dram read+write per layer x layers)",
                      "algorithmic_bytes_per_launch": 2 * 4 * w.B * w.S * w.m_pitch * (w.Lmax - 1),
                      "algorithmic_ops_per_launch": relax_per_launch,
-                     "kernel": "layer_tiled_kernel (one cooperative launch over all layers"
-                               + (", packed 16-bit variant)" if r["packed"] else ")"),
+                     "kernel": ("cluster_search_kernel (one thread-block cluster per instance, all layers in one launch)" if r["cluster"] else
+                                "layer_tiled_kernel (one cooperative launch over all layers"
+                                + (", packed 16-bit variant)" if r["packed"] else ")")),
                      "launch_ms": r["layer_loop_ms"], "launch_ms_min": r["layer_loop_ms_min"],
                      "launch_ms_max": r["layer_loop_ms_max"], "launches_timed": r["layer_loop_launches_timed"],
                      "peak_source": "derived: 148 SMs x 64 int32 lanes x 1.965 GHz, one fused add-min per lane per clock"
@@ -463,6 +476,8 @@ def main():
             o = {key: rk[key] for key in ("ms_per_step", "cells_per_s", "relax_per_s", "searches_per_s")}
             o["alu_frac"] = rk["relax_per_s"] / (ALU_PEAK_GOPS * 1e9 * (2 if rk["packed"] else 1))
             o["packed"] = rk["packed"]
+            o["kernel"] = "cluster" if rk["cluster"] else "tiled"
+            o["layer_loop_ms"] = rk["layer_loop_ms"]
             if k in (1, 2, 4):
                 # with both opt-in flags (work proved unnecessary left out; same tables): no ALU-roofline fraction
                 sbd, rd = bench_workload(torch, galv, wk, max(5, args.steps // 2), 3, barrier,
@@ -472,6 +487,12 @@ def main():
                                         "hbm_frac": 2 * 4 * int(np.sum(wk.L)) * wk.S * pitch4 / (rd["layer_loop_ms"] * 1e-3) / (hbm_gbs * 1e9),
                                         "opt_cost_sum": rd["opt_cost_sum"], "opt_cost_sum_plain": rk["opt_cost_sum"]}
                 del sbd
+            if rk["cluster"]:
+                # the same step on the tiled kernels (what a batch this small ran on before the cluster kernel)
+                sbt, rt = bench_workload(torch, galv, wk, max(5, args.steps // 2), 3, barrier, flags=1 | gb.KERNEL_NO_CLUSTER)
+                o["tiled_kernels_only"] = {"ms_per_step": rt["ms_per_step"], "layer_loop_ms": rt["layer_loop_ms"], "packed": rt["packed"],
+                                           "opt_cost_sum": rt["opt_cost_sum"], "opt_cost_sum_cluster": rk["opt_cost_sum"]}
+                del sbt
             # the same step replayed from a CUDA graph (launch latency matters for the small workloads)
             g = torch.cuda.CUDAGraph()
             s = torch.cuda.Stream()
@@ -486,6 +507,19 @@ def main():
             del sbk, g
             torch.cuda.empty_cache()
         line["others"] = others
+        # One model searched again at run time (the paper's monitoring / optimisation loop): a batch of ONE instance.
+        single = {}
+        for k, inst in ((1, 15), (2, 56)):                       # micro-batch 16 of the GPT-style stack; b = 8, one stage of 96 layers
+            wk = workload_for(k).take([inst])
+            e = {}
+            for key, fl in (("cluster_kernel", 1), ("tiled_kernels_only", 1 | gb.KERNEL_NO_CLUSTER)):
+                sb1, r1 = bench_workload(torch, galv, wk, 50, 5, barrier, flags=fl)
+                e[key] = {"ms_per_step": r1["ms_per_step"], "layer_loop_ms": r1["layer_loop_ms"], "opt_cost_sum": r1["opt_cost_sum"],
+                          "kernel": "cluster" if r1["cluster"] else ("tiled packed" if r1["packed"] else "tiled 32-bit"),
+                          "us_per_layer": r1["layer_loop_ms"] * 1e3 / max(1, wk.Lmax - 1)}
+                del sb1
+            single[f"{wk.name}[instance {inst}]"] = e
+        line["single_instance_research"] = single
         # The argmin-table mode (one launch per layer, at least three ALU operations per relaxation), plain and
         # with dominated rows left out: whole steps on config 4 and on the first 40 layers of config 3
         # (its full argmin + cost tables would not leave room for the other buffers of this run).

@@ -66,6 +66,13 @@ extern "C" {
 #define GALV_KERNEL_NO_PACKED 4096 /* never take the packed 16-bit path (two relaxations per instruction on rebased
                                       costs; taken on its own when S <= 64, S % 4 == 0, no argmin table, all layers in
                                       one launch and every transition entry <= 32767; same results) */
+#define GALV_KERNEL_NO_CLUSTER 16384 /* never take the cluster kernel (small batches: one thread-block cluster per instance,
+                                        the table slice kept in shared memory; taken on its own when the batch has few
+                                        work items per layer for the SMs there are, no argmin table is asked for and the
+                                        slice fits; same results) */
+#define GALV_KERNEL_CLUSTER 32768 /* take the cluster kernel whenever the shape allows it, whatever the batch size */
+#define GALV_CLUSTER_SIZE(n) (((n) & 31) << 16) /* the cluster kernel only with clusters of n CTAs (1..16; by default the size is
+                                                   chosen from the shape, the batch and what the device can hold at once) */
 #define GALV_DEBUG_WITHHOLD_LOAD 2048 /* test hook for the time-out path: one CTA never receives its first stage, every
                                          bounded wait that depends on it runs out (about a second each), status gets
                                          GALV_STATUS_TIMEOUT and the call's results are void; nothing faults or hangs */
@@ -172,9 +179,11 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
                    int32_t* status, void* stream);
 
 /*
- * Which inner loop the most recent galv_dp_search on `workspace` ran: *packed = 1 for the packed
- * 16-bit one (two relaxations per instruction; see GALV_KERNEL_NO_PACKED), 0 for the 32-bit one.
- * The choice is made on the device; this call waits for `stream` and reads it back (host pointer).
+ * Which kernel the most recent galv_dp_search on `workspace` ran: *packed = 1 for the tiled kernel
+ * with the packed 16-bit inner loop (two relaxations per instruction; see GALV_KERNEL_NO_PACKED),
+ * 0 for the tiled kernel with the 32-bit one, 2 for the cluster kernel (32-bit loop; see
+ * GALV_KERNEL_NO_CLUSTER).  The choice between the two inner loops is made on the device; this
+ * call waits for `stream` and reads the answer back (host pointer).
  */
 int galv_dp_search_path(galv_ctx* ctx, const galv_shape* shape, const void* workspace, int32_t* packed, void* stream);
 

@@ -20,6 +20,13 @@ STORE_C_FULL, STORE_ARGMIN, KERNEL_REFERENCE, KERNEL_PER_LAYER, SKIP_INFEASIBLE 
 SKIP_DOMINATED = 8192
 DEBUG_WITHHOLD_LOAD = 2048
 KERNEL_NO_PACKED = 4096
+KERNEL_NO_CLUSTER, KERNEL_CLUSTER = 16384, 32768
+PATH_TILED_32, PATH_TILED_PACKED, PATH_CLUSTER = 0, 1, 2
+
+
+def CLUSTER_SIZE(n: int) -> int:
+    """Flag bits that ask for the cluster kernel with clusters of n CTAs."""
+    return (n & 31) << 16
 TRANS_PER_LAYER = 4
 STATIC_WORKSPACE_BYTES = 1 << 20
 
@@ -207,11 +214,12 @@ class Galv:
     def galv_stage_partition(self, Lm, P, range_opt, cuts, bottleneck):
         self._check(self.lib.galv_stage_partition(self.h, Lm, P, _ptr(range_opt), _ptr(cuts), _ptr(bottleneck), _stream()))
 
-    def galv_dp_search_path(self, shape, workspace) -> bool:
-        """True when the most recent search on this workspace ran the packed 16-bit inner loop."""
+    def galv_dp_search_path(self, shape, workspace) -> int:
+        """Kernel of the most recent search on this workspace: 1 tiled kernel with the packed 16-bit inner loop
+        (truthy, as before), 0 tiled kernel with the 32-bit loop, 2 cluster kernel."""
         out = C.c_int32()
         self._check(self.lib.galv_dp_search_path(self.h, C.byref(shape), _ptr(workspace), C.byref(out), _stream()))
-        return bool(out.value)
+        return int(out.value)
 
     def galv_backtrack(self, shape, L, time_q, mem_q, trans_q, Ct, At, C_last, budget, opt_cost, plan, mem_used, status):
         self._check(self.lib.galv_backtrack(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),

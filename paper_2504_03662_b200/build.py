@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgalv.so")
-SOURCES = ["galv_api.cu", "galv_dp.cu", "galv_backtrack.cu", "galv_costs.cu", "galv_probe.cu", "galv_noalloc.cu", "galv_select.cu", "galv_prune.cu", "galv_graph.cu", "galv_stages.cu", "galv_switch.cu"]
+SOURCES = ["galv_api.cu", "galv_dp.cu", "galv_backtrack.cu", "galv_costs.cu", "galv_probe.cu", "galv_noalloc.cu", "galv_select.cu", "galv_prune.cu", "galv_graph.cu", "galv_stages.cu", "galv_switch.cu", "galv_cluster.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 # The cost model must round every product and sum on its own (no fused multiply-add).

@@ -90,6 +90,7 @@ int galv_create(galv_ctx** out, int device_ordinal)
     cudaGetDevice(&cur);
     if (cur != device_ordinal) cudaSetDevice(device_ordinal);
     e = galv_dp_configure(ctx);
+    if (e == cudaSuccess) e = galv_cluster_configure(ctx);
     for (auto& ev : ctx->pev)
         if (e == cudaSuccess) e = cudaEventCreate(&ev);
     if (cur >= 0 && cur != device_ordinal) cudaSetDevice(cur);
@@ -217,7 +218,7 @@ int galv_dp_search_path(galv_ctx* ctx, const galv_shape* sh, const void* workspa
     cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaMemcpy(flags, static_cast<const char*>(workspace) + w.err, sizeof(flags), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(ctx, "galv_dp_search_path", e);
-    *packed = flags[3] != 0;
+    *packed = flags[3];
     return GALV_OK;
 }
 

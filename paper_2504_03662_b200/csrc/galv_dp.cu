@@ -1581,6 +1581,15 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
 {
     cudaError_t e;
     const int B = a.B, Lmax = a.Lmax, S = a.S;
+    {
+        // Small batches: one cluster per instance, the whole search in one launch (no workspace but the path flag).
+        ClPlan cp;
+        if (galv_cluster_plan(ctx, sh, &cp)) {
+            e = galv_cluster_launch(ctx, sh, cp, a, st);
+            if (e == cudaSuccess) return e;
+            (void)cudaGetLastError();                        // the clusters cannot be placed on this device right now: tiled kernels
+        }
+    }
     e = cudaMemsetAsync(a.scratch, 0, (size_t)4 * (Lmax + 2) * 4, st);      // histogram, fill and work counters
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(a.err, 0, 16, st);

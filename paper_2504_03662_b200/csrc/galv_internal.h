@@ -11,6 +11,7 @@ struct galv_ctx {
     int device;
     int num_sms;
     int smem_optin;      // max dynamic shared memory per block (bytes)
+    int max_cluster;     // largest thread-block cluster the cluster kernel may be launched with (8 portable, 16 where allowed)
     int profiling;       // record an event pair around the layer launches of every search
     int prof_count;      // searches profiled since profiling was switched on
     cudaEvent_t pev[2 * 64];   // ring of event pairs: search k uses pev[2*(k%64)], pev[2*(k%64)+1]
@@ -73,6 +74,24 @@ int galv_set_error(galv_ctx* ctx, int code, const char* text);
 // workspace carve-up (offsets in bytes, all 256-aligned)
 struct WsLayout { size_t order, nactive, scratch, err, minmem_l, ntiles, istart, tcount, front, tile_done, trans_p, roll, total; };
 WsLayout galv_ws_layout(const galv_shape* sh);
+
+// How the cluster kernel (small batches: one thread-block cluster per instance) cuts an instance.
+struct ClPlan {
+    int cl;        // CTAs per cluster
+    int w;         // budget columns per CTA (multiple of 32)
+    int g;         // w / 32
+    int nsg;       // ceil(S / 8)
+    int sp8;       // nsg * 8
+    int tm;        // 32-column groups per warp register tile
+    int nct;       // column tiles per CTA
+    int units;     // nct * nsg work units per CTA and layer
+    int nw;        // warps per CTA
+    int smem;      // dynamic shared memory bytes
+    int sorted;    // clusters take the instances longest first
+};
+bool galv_cluster_plan(const galv_ctx* ctx, const galv_shape* sh, ClPlan* plan);
+cudaError_t galv_cluster_configure(galv_ctx* ctx);
+cudaError_t galv_cluster_launch(galv_ctx* ctx, const galv_shape* sh, const ClPlan& plan, const struct DpArgs& a, cudaStream_t st);
 
 bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* plan);
 cudaError_t galv_dp_configure(const galv_ctx* ctx);

@@ -10,6 +10,12 @@ from paper_2504_03662_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 INF = 2 ** 30 - 1
+NC, CLU = 16384, 32768        # GALV_KERNEL_NO_CLUSTER (tiled kernels only), GALV_KERNEL_CLUSTER (cluster kernel wherever the shape allows)
+
+
+def cl_size(n):
+    """GALV_CLUSTER_SIZE(n): the cluster kernel with clusters of n CTAs."""
+    return CLU | ((n & 31) << 16)
 
 
 @pytest.fixture(scope="module")
@@ -71,9 +77,12 @@ def check_batch(orc, galv, w, flags, idx=None, tables=True, budget=None):
             r = dict(r, opt_cost=o, plan=p, mem_used=u, status=st)
         assert res["status"][i] == r["status"], (i, res["status"][i], r["status"])
         assert res["opt_cost"][i] == r["opt_cost"], i
-        assert (res["plan"][i, :Li] == r["plan"]).all(), (i, res["plan"][i, :Li], r["plan"])
-        assert (res["plan"][i, Li:] == -1).all()
-        assert res["mem_used"][i] == r["mem_used"]
+        if flags & (gb.STORE_C_FULL | gb.STORE_ARGMIN):
+            assert (res["plan"][i, :Li] == r["plan"]).all(), (i, res["plan"][i, :Li], r["plan"])
+            assert (res["plan"][i, Li:] == -1).all()
+            assert res["mem_used"][i] == r["mem_used"]
+        else:                                                   # no table kept: the optimum only, no walk
+            assert (res["plan"][i] == -1).all() and res["mem_used"][i] == 0
         if r["C"] is None:
             continue
         last = sb.C_last[i, :, :w.M + 1].t().cpu().numpy()
@@ -88,8 +97,9 @@ def check_batch(orc, galv, w, flags, idx=None, tables=True, budget=None):
     return sb, res
 
 
-MODES = [1, 3, 2, 1 | 512, 1 | 256, 3 | 256]   # full C (all layers in one launch); full C + A; rolling + A;
-                                             # full C with one launch per layer; the reference kernel
+MODES = [1 | NC, 3, 2, 1 | 512, 1 | 256, 3 | 256, 1, 1 | CLU]   # full C (all layers in one launch); full C + A; rolling + A;
+                                             # full C with one launch per layer; the reference kernel; the cluster
+                                             # kernel (chosen on its own for a batch this small; and asked for)
 
 
 @pytest.mark.parametrize("flags", MODES)
@@ -122,7 +132,8 @@ SHAPES = [  # B, Lmax, S, M, kwargs
 ]
 
 
-@pytest.mark.parametrize("flags", [1, 3, 2, 1 | 512, 1 | 1024, 2 | 1024])
+@pytest.mark.parametrize("flags", [1 | NC, 3, 2, 1 | 512, 1 | 1024 | NC, 2 | 1024, 1 | CLU, 1 | cl_size(2), 1 | cl_size(3), 1 | cl_size(5),
+                                   1 | cl_size(8), 1 | cl_size(16)])
 @pytest.mark.parametrize("k", range(len(SHAPES)))
 def test_random_shapes(orc, galv, flags, k):
     B, Lmax, S, M, kw = SHAPES[k]
@@ -159,13 +170,24 @@ def test_flagged_instances_are_skipped(orc, galv):
 def test_config1_full(orc, galv):
     sb, res = check_batch(orc, galv, inputs.config1(), 3)
     assert (res["status"] == 0).all()
+    # a batch this small takes the cluster kernel on its own
+    sb, res = check_batch(orc, galv, inputs.config1(), 1)
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == 2 and (res["status"] == 0).all()
+    sb, res = check_batch(orc, galv, inputs.config1(), 1 | NC)
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == 0
 
 
 def test_config2_full_ragged(orc, galv):
     w = inputs.config2()
-    sb, res = check_batch(orc, galv, w, 1)
-    assert set(res["status"].tolist()) <= {0, 1}
+    sb, res = check_batch(orc, galv, w, 1 | NC)
+    assert set(res["status"].tolist()) <= {0, 1} and galv.galv_dp_search_path(sb.shape, sb.workspace) == 1
     sb, res = check_batch(orc, galv, w, 2, idx=range(0, 64, 5), tables=False)
+    # the cluster kernel: more instances than cluster slots, the longest first
+    sb, res = check_batch(orc, galv, w, 1 | CLU)
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == 2
+    for n in (6, 16):
+        sb, res = check_batch(orc, galv, w, 1 | cl_size(n), idx=range(0, 64, 3))
+        assert galv.galv_dp_search_path(sb.shape, sb.workspace) == 2
 
 
 def test_config2_full_product_extra(orc, galv):
@@ -200,7 +222,7 @@ def test_config4_full_size_dominated_rows_skipped(orc, galv):
     w = inputs.config4()
     idx = [0, 511, 1023] + list(range(100, 1024, 300))
     sb, res = check_batch(orc, galv, w, gb.STORE_C_FULL | gb.SKIP_DOMINATED, idx=idx)
-    assert not galv.galv_dp_search_path(sb.shape, sb.workspace)
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == 0
     assert (res["status"] == 0).all()
     _properties_all(orc, w, w.time_q, w.mem_q, w.trans_q, sb, res)
 
@@ -304,7 +326,7 @@ def test_alu_probe_runs(galv):
     assert all(1e11 < r < 1e15 for r in rates), rates
 
 
-@pytest.mark.parametrize("flags", [1, 1 | 1024, 1 | 512, 3])
+@pytest.mark.parametrize("flags", [1 | NC, 1 | 1024 | NC, 1 | 512, 3, 1 | CLU])
 def test_layers_with_different_tile_counts(orc, galv, flags):
     """One heavy layer leaves its trailing tiles out; the layers after it run them again.
 
@@ -370,7 +392,8 @@ def test_one_launch_against_reference_kernel_on_many_shapes(galv, block):
             w.mem_q[:, int(rng.integers(1, Lmax)), :] += M // 2       # one heavy layer: fewer tiles there
         ref = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_REFERENCE)
         ref.dp_search()
-        one = SearchBuffers(galv, w, gb.STORE_C_FULL | (gb.SKIP_INFEASIBLE if case % 3 == 2 else 0) | (gb.SKIP_DOMINATED if case % 4 == 1 else 0))
+        one = SearchBuffers(galv, w, gb.STORE_C_FULL | (gb.KERNEL_CLUSTER if case % 5 == 4 else gb.KERNEL_NO_CLUSTER)
+                            | (gb.SKIP_INFEASIBLE if case % 3 == 2 else 0) | (gb.SKIP_DOMINATED if case % 4 == 1 else 0))
         for _ in range(2):
             one.C.fill_(-7)
             one.dp_search()
@@ -392,9 +415,11 @@ def test_soak_random_shapes_and_flags(galv):
     import torch
     from paper_2504_03662_b200 import binding as gb
     from paper_2504_03662_b200.search import SearchBuffers
-    choices = [0, gb.SKIP_INFEASIBLE, gb.SKIP_DOMINATED, gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE, gb.KERNEL_NO_PACKED,
-               gb.KERNEL_NO_PACKED | gb.SKIP_DOMINATED, gb.STORE_ARGMIN, gb.STORE_ARGMIN | gb.SKIP_DOMINATED,
-               gb.KERNEL_PER_LAYER | gb.SKIP_DOMINATED]
+    nc = gb.KERNEL_NO_CLUSTER
+    choices = [nc, nc | gb.SKIP_INFEASIBLE, nc | gb.SKIP_DOMINATED, nc | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE, nc | gb.KERNEL_NO_PACKED,
+               nc | gb.KERNEL_NO_PACKED | gb.SKIP_DOMINATED, gb.STORE_ARGMIN, gb.STORE_ARGMIN | gb.SKIP_DOMINATED,
+               gb.KERNEL_PER_LAYER | gb.SKIP_DOMINATED, 0, gb.KERNEL_CLUSTER, gb.CLUSTER_SIZE(2), gb.CLUSTER_SIZE(4), gb.CLUSTER_SIZE(7),
+               gb.CLUSTER_SIZE(16)]
     for block in range(int(os.environ["GALV_SOAK"])):
         rng = np.random.default_rng(77000 + block)
         for case in range(10):
@@ -450,7 +475,7 @@ def test_kernel_span_statistics(galv):
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("flags", [0, 1024])
+@pytest.mark.parametrize("flags", [NC, 1024 | NC, CLU])
 @pytest.mark.parametrize("k", range(len(SHAPES)))
 def test_cost_only_search_on_the_rolling_buffer(orc, galv, flags, k):
     """No table kept: two layers roll in the workspace (all layers still one launch, an item also waits for
@@ -482,15 +507,16 @@ def test_cost_only_search_many_layers_against_full_table(galv):
                                                 (40, 25, 64, 3000, dict(mem_lo=1, mem_hi=900, ragged=True)),
                                                 (300, 12, 24, 700, dict(mem_lo=0, mem_hi=40, ragged=True))]):
         w = inputs.random_tables(8100 + seed, B, Lmax, S, M, **kw)
-        full = SearchBuffers(galv, w, gb.STORE_C_FULL)
+        full = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_NO_CLUSTER)
         full.dp_search(); full.backtrack()
-        lean = SearchBuffers(galv, w, 0)
-        for _ in range(3):
-            lean.dp_search(); lean.backtrack()
-            torch.cuda.synchronize()
-            assert torch.equal(lean.status, full.status) and torch.equal(lean.opt_cost, full.opt_cost)
-            ok = full.status == 0
-            assert torch.equal(lean.C_last[ok], full.C_last[ok])
+        for lean_flags in (gb.KERNEL_NO_CLUSTER, gb.KERNEL_CLUSTER):
+          lean = SearchBuffers(galv, w, lean_flags)
+          for _ in range(3):
+              lean.dp_search(); lean.backtrack()
+              torch.cuda.synchronize()
+              assert torch.equal(lean.status, full.status) and torch.equal(lean.opt_cost, full.opt_cost)
+              ok = full.status == 0
+              assert torch.equal(lean.C_last[ok], full.C_last[ok])
 
 
 @pytest.mark.parametrize("k", [3, 4])
@@ -553,15 +579,15 @@ def test_packed_16bit_path_choice_and_parity(orc, galv, S, M, B, Lmax):
         w.trans_q[0, 0, min(1, S - 1)] = top                     # the largest entry is really there
         w.time_q[B - 1, 1, :] = 7                                # a cheap layer: big spreads between strategies elsewhere
         w.mem_q[0, 2, : S // 2] = M + 5                          # +inf rows in some columns
-        sb = SearchBuffers(galv, w, gb.STORE_C_FULL)
+        sb = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_NO_CLUSTER)
         sb.dp_search(); sb.backtrack()
         assert galv.galv_dp_search_path(sb.shape, sb.workspace) == want
         res = sb.results()
-        plain = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_NO_PACKED)
+        plain = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_NO_PACKED | gb.KERNEL_NO_CLUSTER)
         plain.dp_search(); plain.backtrack()
         assert not galv.galv_dp_search_path(plain.shape, plain.workspace)
         assert torch.equal(sb.status, plain.status) and torch.equal(sb.opt_cost, plain.opt_cost)
-        pruned = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.SKIP_DOMINATED)     # dominated row pairs left out
+        pruned = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.SKIP_DOMINATED | gb.KERNEL_NO_CLUSTER)     # dominated row pairs left out
         pruned.dp_search(); pruned.backtrack()
         assert galv.galv_dp_search_path(pruned.shape, pruned.workspace) == want
         assert torch.equal(pruned.status, plain.status) and torch.equal(pruned.opt_cost, plain.opt_cost)
@@ -575,7 +601,8 @@ def test_packed_16bit_path_choice_and_parity(orc, galv, S, M, B, Lmax):
             if r["C"] is not None:
                 assert (sb.table(i)[:Li] == r["C"]).all(), (top, i)
     # shapes the packed path does not take: S not a multiple of 4, S > 64, an argmin table
-    for S2, flags in ((6, gb.STORE_C_FULL), (70, gb.STORE_C_FULL), (S, gb.STORE_C_FULL | gb.STORE_ARGMIN)):
+    nc = gb.KERNEL_NO_CLUSTER
+    for S2, flags in ((6, gb.STORE_C_FULL | nc), (70, gb.STORE_C_FULL | nc), (S, gb.STORE_C_FULL | gb.STORE_ARGMIN)):
         w = inputs.random_tables(77, 2, 4, S2, 200, trans_hi=100)
         sb = SearchBuffers(galv, w, flags)
         sb.dp_search()
@@ -603,7 +630,7 @@ def test_dominated_rows_left_out(orc, galv, S, M, trans_hi, time_hi):
                   gb.STORE_C_FULL | gb.STORE_ARGMIN | gb.SKIP_DOMINATED,                # one launch per layer, argmin table
                   gb.STORE_ARGMIN | gb.SKIP_DOMINATED | gb.SKIP_INFEASIBLE,
                   gb.STORE_C_FULL | gb.KERNEL_PER_LAYER | gb.SKIP_DOMINATED):
-        sb = SearchBuffers(galv, w, flags)
+        sb = SearchBuffers(galv, w, flags | gb.KERNEL_NO_CLUSTER)
         sb.dp_search(); sb.backtrack()
         packable = (S % 4 == 0 and int(w.trans_q.max()) <= 32767
                     and not flags & (gb.KERNEL_NO_PACKED | gb.STORE_ARGMIN | gb.KERNEL_PER_LAYER))
@@ -633,9 +660,9 @@ def test_packed_path_with_costs_near_the_limit(orc, galv):
     w.time_q[1, 2, ::2] = 0                                              # and some spread between strategies
     w.mem_q[2, 1, :] = M + 1                                             # instance 2: nothing fits from layer 1 on
     assert orc.validate(w.time_q[0], w.mem_q[0], w.trans_q[0]) == 0
-    sb = SearchBuffers(galv, w, gb.STORE_C_FULL)
+    sb = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_NO_CLUSTER)
     sb.dp_search(); sb.backtrack()
-    assert galv.galv_dp_search_path(sb.shape, sb.workspace)
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == 1
     res = sb.results()
     for i in range(B):
         r = orc.search(w.time_q[i], w.mem_q[i], w.trans_q[i], M)
@@ -645,15 +672,17 @@ def test_packed_path_with_costs_near_the_limit(orc, galv):
     assert res["status"][2] == 1 and res["opt_cost"][2] == INF
 
 
-def test_two_streams_at_once(orc, galv):
+@pytest.mark.parametrize("cluster", [NC, CLU])
+def test_two_streams_at_once(orc, galv, cluster):
     """Two searches enqueued on two streams, each with its own workspace: the one-launch kernels take turns on
-    the GPU (a cooperative launch needs all its CTAs resident); both must finish and be right."""
+    the GPU (a cooperative launch needs all its CTAs resident), the cluster kernels share it; both must finish
+    and be right."""
     import torch
     from paper_2504_03662_b200 import binding as gb
     from paper_2504_03662_b200.search import SearchBuffers
     wa = inputs.random_tables(501, 40, 20, 32, 2000, mem_lo=1, mem_hi=150, trans_hi=900)       # packed loop
     wb = inputs.random_tables(502, 30, 25, 24, 1500, mem_lo=1, mem_hi=100, trans_hi=60000)     # 32-bit loop
-    sa, sb_ = SearchBuffers(galv, wa, gb.STORE_C_FULL), SearchBuffers(galv, wb, gb.STORE_C_FULL)
+    sa, sb_ = SearchBuffers(galv, wa, gb.STORE_C_FULL | cluster), SearchBuffers(galv, wb, gb.STORE_C_FULL | cluster)
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
     torch.cuda.synchronize()
     for _ in range(3):
@@ -668,3 +697,83 @@ def test_two_streams_at_once(orc, galv):
             r = orc.search(w.time_q[i], w.mem_q[i], w.trans_q[i], w.M)
             assert res["status"][i] == r["status"] and res["opt_cost"][i] == r["opt_cost"]
             assert (res["plan"][i] == r["plan"]).all() and (s.table(i) == r["C"]).all()
+
+
+@pytest.mark.parametrize("n,M", [(1, 1000), (2, 1000), (3, 1000), (4, 1000), (5, 1000), (6, 2880), (7, 2880), (8, 2880), (9, 2880),
+                                 (12, 2880), (16, 2880)])
+def test_cluster_kernel_every_cluster_size(orc, galv, n, M):
+    """One shape cut over clusters of 1 .. 16 CTAs: columns per CTA, tiles that straddle two CTAs, pushes that skip
+    a whole CTA (mem larger than a CTA's columns) and strategies that never fit all change with the size."""
+    from paper_2504_03662_b200 import binding as gb
+    w = inputs.random_tables(600 + n, 5, 7, 24, M, ragged=True, mem_lo=0, mem_hi=700, trans_hi=40000)
+    w.mem_q[1, 2, :5] = M + 1                                  # never fits
+    w.mem_q[2, 1, :] = 0                                       # a layer that costs no memory
+    w.mem_q[3, 3, 4] = M                                       # fits only at the very edge
+    sb, res = check_batch(orc, galv, w, gb.STORE_C_FULL | gb.CLUSTER_SIZE(n))
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == gb.PATH_CLUSTER
+    # without a table: only the last layer and the optimum
+    sb, res = check_batch(orc, galv, w, gb.CLUSTER_SIZE(n))
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == gb.PATH_CLUSTER
+
+
+def test_cluster_kernel_more_instances_than_cluster_slots(orc, galv):
+    """Hundreds of ragged instances: clusters are handed the instances longest first; every instance is searched
+    exactly once, flagged ones are reported and skipped.  Above 512 instances the tiled kernels take over."""
+    from paper_2504_03662_b200 import binding as gb
+    for B, want in ((400, gb.PATH_CLUSTER), (512, gb.PATH_CLUSTER), (600, None)):
+        w = inputs.random_tables(8800 + B, B, 6, 8, 1000, ragged=True, mem_lo=0, mem_hi=300)
+        w.time_q[7, 0, 0] = -1
+        w.L[11] = 0
+        w.L[13] = 7
+        w.time_q[17] = (INF - 1) // 2
+        w.L[17] = 3
+        sb, res = check_batch(orc, galv, w, gb.STORE_C_FULL | gb.CLUSTER_SIZE(8), idx=[0, 1, 2, 7, 17, B // 2, B - 1] + list(range(20, B, 37)))
+        path = galv.galv_dp_search_path(sb.shape, sb.workspace)
+        assert path == want if want is not None else path != gb.PATH_CLUSTER
+        assert res["status"][[7, 11, 13, 17]].tolist() == [2, 2, 2, 4]
+        # the rest against the tiled kernel, cell by cell
+        ref = __import__("paper_2504_03662_b200.search", fromlist=["SearchBuffers"]).SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_NO_CLUSTER)
+        ref.dp_search(); ref.backtrack()
+        import torch
+        torch.cuda.synchronize()
+        assert torch.equal(ref.status, sb.status) and torch.equal(ref.opt_cost, sb.opt_cost) and torch.equal(ref.plan, sb.plan)
+        ok = ref.status == 0
+        assert torch.equal(ref.C_last[ok], sb.C_last[ok])
+        for i in np.flatnonzero(ok.cpu().numpy()):
+            Li = int(w.L[i])
+            assert torch.equal(ref.C[i, :Li], sb.C[i, :Li]), int(i)
+
+
+def test_cluster_kernel_flagged_instances(orc, galv):
+    """Validation inside the cluster kernel: the same verdicts as the validation pass of the tiled path."""
+    from paper_2504_03662_b200 import binding as gb
+    w = inputs.random_tables(5, 6, 4, 6, 50, ragged=True)
+    w.time_q[1, 0, 2] = -7
+    w.L[2] = 0
+    w.time_q[3] = (INF - 1) // 2
+    w.L[3] = 4
+    w.mem_q[4, 1, :] = -1
+    w.L[4] = 4
+    w.L[5] = 9
+    w.trans_q[0, 1, 2] = 0
+    sb, res = check_batch(orc, galv, w, gb.STORE_C_FULL | gb.KERNEL_CLUSTER, idx=[0])
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == gb.PATH_CLUSTER
+    assert res["status"].tolist()[1:] == [2, 2, 4, 2, 2]
+    assert (res["opt_cost"][1:] == INF).all() and (res["plan"][1:] == -1).all()
+    w.trans_q[0, 1, 2] = -1                                    # a negative transition entry
+    sb, res = check_batch(orc, galv, w, gb.STORE_C_FULL | gb.KERNEL_CLUSTER, idx=[])
+    assert res["status"][0] == 2
+
+
+def test_cluster_kernel_is_chosen_for_small_batches_only(galv):
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    for w, want in ((inputs.config0(), gb.PATH_CLUSTER), (inputs.config4(B=16), gb.PATH_CLUSTER),
+                    (inputs.config4(B=700), gb.PATH_TILED_32)):
+        sb = SearchBuffers(galv, w, gb.STORE_C_FULL)
+        sb.dp_search()
+        assert galv.galv_dp_search_path(sb.shape, sb.workspace) == want, w.B
+    # an argmin table keeps the tiled kernels, whatever the flag asks
+    sb = SearchBuffers(galv, inputs.config0(), gb.STORE_C_FULL | gb.STORE_ARGMIN | gb.KERNEL_CLUSTER)
+    sb.dp_search()
+    assert galv.galv_dp_search_path(sb.shape, sb.workspace) == gb.PATH_TILED_32

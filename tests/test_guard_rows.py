@@ -61,7 +61,8 @@ def guarded_buffers(galv, w, flags):
     return sb, guards
 
 
-MODES = [1, 3, 2, 0, 1 | 512, 1 | 1024 | 8192, 1 | 4096, 2 | 8192, 1 | 256]
+NC, CLU = 16384, 32768        # tiled kernels only / the cluster kernel wherever the shape allows
+MODES = [1 | NC, 3, 2, NC, 1 | 512, 1 | 1024 | 8192 | NC, 1 | 4096 | NC, 2 | 8192, 1 | 256, 1 | CLU, CLU, 1 | CLU | (2 << 16), 1 | CLU | (16 << 16)]
 
 
 @pytest.mark.parametrize("flags", MODES)
