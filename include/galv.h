@@ -67,12 +67,14 @@ extern "C" {
                                       costs; taken on its own when S <= 64, S % 4 == 0, no argmin table, all layers in
                                       one launch and every transition entry <= 32767; same results) */
 #define GALV_KERNEL_NO_CLUSTER 16384 /* never take the cluster kernel (small batches: one thread-block cluster per instance,
-                                        the table slice kept in shared memory; taken on its own when the batch has few
-                                        work items per layer for the SMs there are, no argmin table is asked for and the
-                                        slice fits; same results) */
-#define GALV_KERNEL_CLUSTER 32768 /* take the cluster kernel whenever the shape allows it, whatever the batch size */
-#define GALV_CLUSTER_SIZE(n) (((n) & 31) << 16) /* the cluster kernel only with clusters of n CTAs (1..16; by default the size is
-                                                   chosen from the shape, the batch and what the device can hold at once) */
+                                        the table slice kept in shared memory; taken on its own when the device can hold
+                                        one cluster per instance at once, no argmin table is asked for, S <= 128 and the
+                                        slice fits in shared memory; same results) */
+#define GALV_KERNEL_CLUSTER 32768 /* take the cluster kernel whenever the shape allows it, also for batches that need
+                                     several rounds of clusters (at most 512 instances then) */
+#define GALV_CLUSTER_SIZE(n) (((n) & 31) << 16) /* the cluster kernel with clusters of n CTAs (1..16), where that size is possible
+                                                   for the shape (by default the size is chosen from the shape, the batch
+                                                   and what the device can hold at once) */
 #define GALV_DEBUG_WITHHOLD_LOAD 2048 /* test hook for the time-out path: one CTA never receives its first stage, every
                                          bounded wait that depends on it runs out (about a second each), status gets
                                          GALV_STATUS_TIMEOUT and the call's results are void; nothing faults or hangs */

@@ -34,6 +34,7 @@ namespace {
 
 constexpr int kInf = GALV_INF;
 constexpr int kMaxSortedB = 512;          // instances whose lengths fit the ranking scratch below
+constexpr int kRowsPerLane = 4;           // strategies per lane of the service warp: S <= 128
 
 struct ClArgs {
     int B, Lmax, S, M, m_pitch;
@@ -128,7 +129,7 @@ __device__ __forceinline__ int fill_count(bool real, int mem, int M, int W, int 
 // is the service warp: it sends the finished layer to the table (one tensor-map store), prepares the next
 // layer's records and, with one matrix per layer, fetches the next matrix.
 template <int TM>
-__global__ void __launch_bounds__(544, 1) cluster_search_kernel(const ClArgs a, const __grid_constant__ CUtensorMap map_c,
+__global__ void __launch_bounds__(416, 1) cluster_search_kernel(const ClArgs a, const __grid_constant__ CUtensorMap map_c,
                                                                 const __grid_constant__ CUtensorMap map_last)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -146,7 +147,9 @@ __global__ void __launch_bounds__(544, 1) cluster_search_kernel(const ClArgs a, 
     const int tmat = S * SP8;
     const int nrec = a.nct * SP8;
     int4* const rows = reinterpret_cast<int4*>(tsm + (a.trans_layer ? 2 : 1) * tmat);     // [2][nct][SP8] push records
-    int* const fillc = reinterpret_cast<int*>(rows + 2 * nrec);                            // [2][SP8]
+    int* const fillc = reinterpret_cast<int*>(rows + 2 * nrec);                            // [2][SP8] leading cells of each row to fill with +inf
+    int* const fillmax = fillc + 2 * SP8;                                                  // [2] the largest of them (padded to 4 ints)
+    int32_t* const dump = fillmax + 4;                                                     // [32 * TM] where stores of skipped strategies go
 
     if (blockIdx.x == 0 && tid == 0) { a.path[0] = 0; a.path[3] = 2; }      // no error flag to raise; the cluster kernel ran
 
@@ -223,20 +226,38 @@ __global__ void __launch_bounds__(544, 1) cluster_search_kernel(const ClArgs a, 
     const int col_g0 = rank * W;                               // first budget column of this CTA
 
     // ---- layer 0, the records of layer 1, the transition matrix
-    // the records and fill counts of layer `lay` into half `h` of the two arrays (threads t, t + nt, ...)
-    auto prepare = [&](int lay, int h, int t, int nt) {
-        for (int s = t; s < SP8; s += nt) {
-            const bool real = s < S;
-            const int mem = real ? mq[lay * S + s] : 0, time = real ? tq[lay * S + s] : 0;
-            fillc[h * SP8 + s] = fill_count(real, mem, M, W, rank);
-            for (int ct = 0; ct < a.nct; ++ct) {
-                const int left = a.G - ct * TM;
-                rows[h * nrec + ct * SP8 + s] = tile_record(real, mem, time, M, W, rank, ct * 32 * TM, 32 * (left < TM ? left : TM));
-            }
+    // the push records and fill count of strategy s (raw mem / time given) into half `h` of the two arrays
+    auto prepare_one = [&](int h, int s, int mem, int time) -> int {                       // returns the row's fill count
+        const bool real = s < S;
+        const int nf = fill_count(real, mem, M, W, rank);
+        fillc[h * SP8 + s] = nf;
+        for (int ct = 0; ct < a.nct; ++ct) {
+            const int left = a.G - ct * TM;
+            rows[h * nrec + ct * SP8 + s] = tile_record(real, mem, time, M, W, rank, ct * 32 * TM, 32 * (left < TM ? left : TM));
         }
+        return nf;
     };
-    prepare(0, 0, tid, NT);
-    if (Li > 1) prepare(1, 1, tid, NT);
+    // ... of a whole layer by one warp: lane k takes strategies k, k+32, ...
+    auto prepare_layer = [&](int h, const int (&m)[kRowsPerLane], const int (&t)[kRowsPerLane]) {
+        int most = 0;
+#pragma unroll
+        for (int j = 0; j < kRowsPerLane; ++j)
+            if (lane + 32 * j < SP8) most = max(most, prepare_one(h, lane + 32 * j, m[j], t[j]));
+        most = __reduce_max_sync(0xffffffffu, most);
+        if (lane == 0) fillmax[h] = most;
+    };
+    // layers 0 and 1 straight from global memory, a warp each (nothing is being stored yet)
+    if (warp <= 1 && warp < Li) {
+        int m0[kRowsPerLane], t0[kRowsPerLane];
+#pragma unroll
+        for (int j = 0; j < kRowsPerLane; ++j) {
+            const int s = lane + 32 * j;
+            m0[j] = s < S ? mq[warp * S + s] : 0;
+            t0[j] = s < S ? tq[warp * S + s] : 0;
+        }
+        prepare_layer(warp, m0, t0);
+    }
+    for (int x = tid; x < 32 * TM; x += NT) dump[x] = 0;
     {
         const int32_t* T = T0 + (a.trans_layer ? a.trans_layer : 0);       // matrix 1 is paid between layers 0 and 1
         int32_t* dst = tsm + (a.trans_layer ? tmat : 0);                    // per layer: matrix l sits in tsm[l & 1]
@@ -248,13 +269,27 @@ __global__ void __launch_bounds__(544, 1) cluster_search_kernel(const ClArgs a, 
     }
     __syncthreads();
     for (int s = warp; s < S; s += NW + 1) {
-        const int t0 = rows[s].z, nf = fillc[s];                            // time(0,s) sits in every record of s
+        const int t0 = rows[s].z;                                           // time(0,s) sits in every record of s
+        const int nf = fillc[s];
         for (int x = lane; x < W; x += 32) {
             const bool pad = col_g0 + x > M;
             buf0[s * W + x] = (pad || x < nf) ? kInf : t0;
             if (pad) buf1[s * W + x] = kInf;                                // pad columns are never written again
         }
     }
+    // Service warp: raw mem / time rows of the layer after next, lane k keeps strategies k, k+32, ... (S <= 128).
+    // They are fetched a whole layer before they are needed and BEFORE that layer's table store is issued: a
+    // global load issued while the SM's bulk stores are in flight comes back after thousands of cycles.
+    int raw_m[kRowsPerLane], raw_t[kRowsPerLane];
+    auto fetch_rows = [&](int lay, int (&m)[kRowsPerLane], int (&t)[kRowsPerLane]) {
+#pragma unroll
+        for (int j = 0; j < kRowsPerLane; ++j) {
+            const int s = lane + 32 * j;
+            m[j] = s < S ? mq[lay * S + s] : 0;
+            t[j] = s < S ? tq[lay * S + s] : 0;
+        }
+    };
+    if (warp == NW && Li > 2) fetch_rows(2, raw_m, raw_t);
     // every CTA of the cluster has started and holds its layer 0 before anyone writes into a neighbour
     cluster_barrier();
 
@@ -266,38 +301,43 @@ __global__ void __launch_bounds__(544, 1) cluster_search_kernel(const ClArgs a, 
 
         if (warp == NW) {
             // ------------------------------------------------------------ service warp
+            // first the loads: rows of layer l+2, and with one matrix per layer the matrix of layer l+1
+            int next_m[kRowsPerLane], next_t[kRowsPerLane];
+            if (l + 2 < Li) fetch_rows(l + 2, next_m, next_t);
+            if (l + 1 < Li && a.trans_layer) {
+                const int32_t* T = T0 + (size_t)(l + 1) * a.trans_layer;
+                int32_t* dst = tsm + (((l + 1) & 1) ? tmat : 0);
+                for (int e = lane; e < S * S; e += 32) {
+                    const int k = e / S, c = e - k * S;
+                    cp_async_4(dst + k * SP8 + c, T + e);
+                }
+            }
             // layer l-1 is complete in X: to the table while this layer is computed
             if (a.C && lane == 0) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // the buffer was written by plain stores
                 tensor_store_3d(&map_c, X, rank * a.G, (i * Lmax + (l - 1)) * S);
                 bulk_commit();
             }
-            // cells of this CTA's columns that no column maps to in this layer
-            for (int s0 = 0; s0 < S; s0 += 32) {
-                const int mine = s0 + lane < S ? fillc[(l & 1) * SP8 + s0 + lane] : 0;
-                unsigned todo = __ballot_sync(0xffffffffu, mine > 0);
-                while (todo) {
-                    const int b = __ffs(todo) - 1;
-                    todo &= todo - 1;
-                    const int n = __shfl_sync(0xffffffffu, mine, b);
-                    for (int x = lane; x < n; x += 32) Y[(s0 + b) * W + x] = kInf;
-                }
-            }
-            if (l + 1 < Li) {
-                prepare(l + 1, (l + 1) & 1, lane, 32);
-                if (a.trans_layer) {
-                    const int32_t* T = T0 + (size_t)(l + 1) * a.trans_layer;
-                    int32_t* dst = tsm + (((l + 1) & 1) ? tmat : 0);
-                    for (int e = lane; e < S * S; e += 32) {
-                        const int k = e / S, c = e - k * S;
-                        cp_async_4(dst + k * SP8 + c, T + e);
-                    }
-                    cp_async_wait_all();
-                }
-            }
+            // the records of layer l+1 from the rows fetched a layer ago
+            if (l + 1 < Li) prepare_layer((l + 1) & 1, raw_m, raw_t);
+#pragma unroll
+            for (int j = 0; j < kRowsPerLane; ++j) { raw_m[j] = next_m[j]; raw_t[j] = next_t[j]; }
+            if (l + 1 < Li && a.trans_layer) cp_async_wait_all();
             if (a.C && lane == 0) bulk_wait_read();                         // X may be overwritten from the next barrier on
         } else {
             // ------------------------------------------------------------ compute warps
+            // cells of this CTA's columns that no column maps to in this layer (m < mem(l,s): the first fillc[s] of
+            // row s): the compute warps share the columns, each takes every strategy in turn (independent predicated
+            // stores; a loop per strategy would be a chain of dependent steps)
+            {
+                const int* const fc = fillc + (l & 1) * SP8;
+                const int most = fillmax[l & 1];
+                for (int x = warp * 32 + lane; x < most; x += NW * 32) {
+#pragma unroll 4
+                    for (int s = 0; s < S; ++s)
+                        if (x < fc[s]) Y[s * W + x] = kInf;
+                }
+            }
             const uint32_t ybase = smem_addr(Y);
             for (int unit = warp; unit < a.units; unit += NW) {
                 const int ct = unit / a.NSG, sg = unit - ct * a.NSG;
@@ -334,48 +374,60 @@ __global__ void __launch_bounds__(544, 1) cluster_search_kernel(const ClArgs a, 
                 };
                 steps(std::integral_constant<int, 8>());
                 steps(std::integral_constant<int, 1>());
-                // push: column m' of strategy s belongs at column m' + mem(l,s): in this CTA's buffer or in one further up
-                const int4* const rt = rl + ct * SP8 + sg * 8;
+                // push: column m' of strategy s belongs at column m' + mem(l,s): in this CTA's buffer or in one further up.
+                // All eight records first; when every strategy either stays at home in one piece or lands nowhere, the
+                // stores go out in one run without a branch (those that land nowhere go to a dump row).
+                int4 r[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) r[u] = rl[ct * SP8 + sg * 8 + u];
+                bool plain = nj == TM;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) plain = plain && (r[u].x < 0 || (r[u].x == rank && r[u].w == kWholeTile));
                 int32_t* const yl = Y + (sg * 8) * W + lane;
+                if (plain) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int4 r = rt[u];
-                    if (r.x < 0) continue;                                  // nothing of this tile lands inside the budget
-                    if (r.w == kWholeTile) {
-                        if (r.x == rank) {
-                            // this CTA's own columns: plain shared-memory stores
-                            int32_t* y = yl + u * W + r.y;
+                    for (int u = 0; u < 8; ++u) {
+                        int32_t* const y = r[u].x < 0 ? dump + lane : yl + u * W + r[u].y;
 #pragma unroll
-                            for (int j = 0; j < TM; ++j)
-                                if (j < nj) y[j * 32] = __viaddmin_s32(acc[j][u], r.z, kInf);            // +inf stays +inf
-                        } else {
-                            const uint32_t ra = map_to_rank(ybase + (uint32_t)((sg * 8 + u) * W + r.y + lane) * 4u, (uint32_t)r.x);
+                        for (int j = 0; j < TM; ++j) y[j * 32] = __viaddmin_s32(acc[j][u], r[u].z, kInf);    // +inf stays +inf
+                    }
+                } else {
 #pragma unroll
-                            for (int j = 0; j < TM; ++j)
-                                if (j < nj) st_cluster(ra + j * 128u, __viaddmin_s32(acc[j][u], r.z, kInf));
-                        }
-                    } else {
-                        // the tile straddles two CTAs or the edge of the budget: every column is checked.  What stays at
-                        // home goes by plain stores; only what crosses to another CTA takes the cluster window.
+                    for (int u = 0; u < 8; ++u) {
+                        if (r[u].x < 0) continue;                           // nothing of this tile lands inside the budget
+                        const bool home = r[u].x == rank;
                         const uint32_t row = ybase + (uint32_t)((sg * 8 + u) * W) * 4u;
-                        const bool home = r.x == rank;
-                        const uint32_t ra0 = home ? 0u : map_to_rank(row, (uint32_t)r.x);
-                        const uint32_t ra1 = map_to_rank(row, (uint32_t)min(r.x + 1, CL - 1)) - (uint32_t)W * 4u;
-                        int32_t* const y = yl + u * W + r.y;
+                        int32_t* const y = yl + u * W + r[u].y;
+                        if (r[u].w == kWholeTile) {
+                            // all of it in one CTA's columns
+                            const uint32_t ra = home ? 0u : map_to_rank(row + (uint32_t)(r[u].y + lane) * 4u, (uint32_t)r[u].x);
 #pragma unroll
-                        for (int j = 0; j < TM; ++j)
-                            if (j < nj) {
-                                const int x = r.y + j * 32 + lane;
-                                const int v = __viaddmin_s32(acc[j][u], r.z, kInf);
-                                if (x <= r.w) {
-                                    if (x < W) {
-                                        if (home) y[j * 32] = v;
-                                        else st_cluster(ra0 + (uint32_t)x * 4u, v);
-                                    } else {
-                                        st_cluster(ra1 + (uint32_t)x * 4u, v);
+                            for (int j = 0; j < TM; ++j)
+                                if (j < nj) {
+                                    const int v = __viaddmin_s32(acc[j][u], r[u].z, kInf);
+                                    if (home) y[j * 32] = v;
+                                    else st_cluster(ra + j * 128u, v);
+                                }
+                        } else {
+                            // the tile straddles two CTAs or the edge of the budget: every column is checked.  What stays
+                            // at home goes by plain stores; only what crosses to another CTA takes the cluster window.
+                            const uint32_t ra0 = home ? 0u : map_to_rank(row, (uint32_t)r[u].x);
+                            const uint32_t ra1 = map_to_rank(row, (uint32_t)min(r[u].x + 1, CL - 1)) - (uint32_t)W * 4u;
+#pragma unroll
+                            for (int j = 0; j < TM; ++j)
+                                if (j < nj) {
+                                    const int x = r[u].y + j * 32 + lane;
+                                    const int v = __viaddmin_s32(acc[j][u], r[u].z, kInf);
+                                    if (x <= r[u].w) {
+                                        if (x < W) {
+                                            if (home) y[j * 32] = v;
+                                            else st_cluster(ra0 + (uint32_t)x * 4u, v);
+                                        } else {
+                                            st_cluster(ra1 + (uint32_t)x * 4u, v);
+                                        }
                                     }
                                 }
-                            }
+                        }
                     }
                 }
             }
@@ -493,22 +545,27 @@ bool galv_cluster_plan(const galv_ctx* ctx, const galv_shape* sh, ClPlan* out)
     if (sh->flags & (GALV_STORE_ARGMIN | GALV_KERNEL_REFERENCE | GALV_KERNEL_PER_LAYER | GALV_DEBUG_WITHHOLD_LOAD | GALV_KERNEL_NO_CLUSTER))
         return false;
     const int S = sh->S, Gt = sh->m_pitch / 32;
+    if (S > 32 * kRowsPerLane) return false;
     if ((long long)sh->B * sh->Lmax * S >= (1ll << 31)) return false;       // row coordinates of the table store are 32-bit
     const int nsg = (S + 7) / 8, sp8 = nsg * 8;
     const int nT = (sh->flags & GALV_TRANS_PER_LAYER) ? 2 : 1;
     const int budget = ctx->smem_optin - 4096;               // static shared memory of the kernel, rounded up
     // Candidates: every cluster size that gives each CTA at least 96 columns and leaves none without columns.
-    // Estimated time of the batch, in SM cycles per layer: rounds of clusters (all instances taken as equally
-    // long) x (a CTA's add-min issue time + what a layer costs besides: push, barrier, start).  A larger cluster
-    // shortens every instance's own chain of layers, which is what counts when the lengths differ, so a smaller
-    // one must be clearly better to win.
+    // Estimated SM cycles per layer of a cluster, fitted to measurements on B200: the add-min issue time of the
+    // busiest scheduler, stretched by the per-cell work beside it (push, fill, shared-memory loads: about 24
+    // add-mins' worth per cell), plus what a layer costs whatever its size (barrier, drain of the pushes that
+    // cross CTAs, start): about 3000 cycles, some more for clusters beyond 12 CTAs.  With more instances than the
+    // device holds clusters the batch takes several rounds; on its own the kernel is chosen only when one round
+    // does (a batch that needs rounds is better off on the tiled kernels, whose SMs never wait on a barrier).
     double best_time = 0.0;
     bool found = false;
     const int want_cl = (sh->flags >> 16) & 31;              // GALV_CLUSTER_SIZE(n): only clusters of n CTAs
+    const bool forced = (sh->flags & GALV_KERNEL_CLUSTER) != 0 || want_cl != 0;
     for (int cl = ctx->max_cluster; cl >= 1; --cl) {
+        if (want_cl && cl != want_cl) continue;
         const int g = (Gt + cl - 1) / cl;
         if (cl > 1 && (g < 3 || g * (cl - 1) >= Gt)) continue;
-        const long long smem = (long long)2 * S * g * 32 * 4 + (long long)nT * S * sp8 * 4 + (long long)2 * ((g + 1) / 2) * sp8 * 16 + (long long)2 * sp8 * 4;
+        const long long smem = (long long)2 * S * g * 32 * 4 + (long long)nT * S * sp8 * 4 + (long long)2 * ((g + 1) / 2) * sp8 * 16 + (long long)2 * sp8 * 4 + 16 + 512;
         if (smem > budget) break;                            // smaller clusters need more per CTA
         ClPlan p;
         std::memset(&p, 0, sizeof(p));
@@ -516,17 +573,17 @@ bool galv_cluster_plan(const galv_ctx* ctx, const galv_shape* sh, ClPlan* out)
         const int cost = tile_cost(g, nsg, &p.tm);
         p.nct = (g + p.tm - 1) / p.tm;
         p.units = p.nct * nsg;
-        p.nw = (p.units + 3) & ~3;
-        if (p.nw > 16) p.nw = 16;
+        p.nw = (p.units + 3) & ~3;                           // a multiple of 4: the SM's four schedulers get the same share
+        if (p.nw > 12) p.nw = 12;
         p.smem = (int)smem;
         const int slots = max_active_clusters(ctx, p);
         if (slots < 1) continue;
-        if (want_cl && cl != want_cl) continue;
+        if (!forced && sh->B > slots) continue;
         const double rounds = (double)((sh->B + slots - 1) / slots);
         const double active = (double)(sh->B < slots ? sh->B : slots) * cl;     // CTAs resident at once
         const double share = active > ctx->num_sms ? active / ctx->num_sms : 1.0;   // ... of which this many share an SM's ALUs
-        const double t = rounds * ((double)cost * 16.0 * S * share + 1500.0);
-        if (!found || t < 0.85 * best_time) {
+        const double t = rounds * ((double)cost * 16.0 * S * (1.0 + 24.0 / S) * share + 3000.0 + (cl > 12 ? 800.0 : 0.0));
+        if (!found || t < best_time) {
             best_time = t;
             found = true;
             p.sorted = sh->B > slots;                        // more clusters than fit at once: the longest instances first
@@ -535,13 +592,7 @@ bool galv_cluster_plan(const galv_ctx* ctx, const galv_shape* sh, ClPlan* out)
     }
     if (!found) return false;
     if (out->sorted && sh->B > kMaxSortedB) return false;
-    if (sh->flags & GALV_KERNEL_CLUSTER) return true;
-    // On its own only where the tiled kernel would be a chain of dependent layers: few work items per layer
-    // (instance x tile of >= 128 columns x block of <= 64 strategies) for the SMs there are.
-    DpPlan dp;
-    if (!galv_dp_make_plan(ctx, sh, &dp)) return true;
-    const long long items = (long long)sh->B * dp.ntiles_m * dp.nsb;
-    return items < (long long)6 * ctx->num_sms;
+    return true;
 }
 
 cudaError_t galv_cluster_configure(galv_ctx* ctx)
