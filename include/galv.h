@@ -131,7 +131,13 @@ const char* galv_last_error(const galv_ctx* ctx);
  * shared row with layer_stride_B = 0; strat [S]; inst [B].
  * time_s, mem_bytes [B][Lmax][S] may be NULL.  Entries of layers l >= L[i] are left untouched.
  * status[i] is set to 0, or GALV_STATUS_BAD_INPUT when L[i] is outside 1..Lmax
- * (nothing is written for that instance).
+ * (nothing is written for that instance) or when a descriptor is one no profiler
+ * could have produced: an instance parameter, h, seq or batch_div that is not a
+ * positive finite number, a negative or non-finite layer coefficient, tp or dp
+ * below 1, a ZeRO stage outside 0..3, ckpt or sp other than 0/1.  Such an
+ * instance (every instance, when the strategy table is at fault) gets -1 in all
+ * its time_q, mem_q and trans_q entries, which galv_dp_search flags in turn;
+ * its time_s / mem_bytes are left untouched.
  */
 int galv_eval_costs(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
                     const galv_layer_desc* layers, int64_t layer_stride_B,

@@ -268,10 +268,42 @@ int32_t orc_quant_mem(double bytes, double bin_bytes)
     return (int32_t)q;
 }
 
-/* One instance: every (layer, strategy) and every (s', s). Outputs may be NULL. */
-void orc_eval_costs(int L, int S, const orc_layer *layers, const orc_strategy *strat, const orc_inst *in,
-                    double *time_s, double *mem_bytes, int32_t *time_q, int32_t *mem_q, int32_t *trans_q)
+/* Descriptors the profilers cannot have produced (the paper's model, hardware and dataset profilers report
+ * sizes, rates and counts: Section 3): a rate, size or divisor that is not a positive finite number, a degree
+ * below 1, a ZeRO stage outside 0..3, a flag that is not 0/1, a negative coefficient.  An instance with any such
+ * descriptor among its own parameters, the strategy table or its L layers is flagged ORC_BAD_INPUT as a whole. */
+static int pos_finite(double x) { return x > 0.0 && x < INFINITY; }
+static int nonneg_finite(double x) { return x >= 0.0 && x < INFINITY; }
+int orc_check_descriptors(int L, int S, const orc_layer *layers, const orc_strategy *strat, const orc_inst *in)
 {
+    int ok = pos_finite(in->b) && pos_finite(in->act_mult) && pos_finite(in->flops_rate) && pos_finite(in->bw_tp) &&
+             pos_finite(in->bw_dp) && pos_finite(in->bytes_per_elem) && pos_finite(in->bin_bytes) && pos_finite(in->time_unit_ns);
+    for (int s = 0; s < S; s++)
+        ok = ok && strat[s].tp >= 1 && strat[s].dp >= 1 && strat[s].zero >= 0 && strat[s].zero <= 3 &&
+             (strat[s].ckpt == 0 || strat[s].ckpt == 1) && (strat[s].sp == 0 || strat[s].sp == 1) && pos_finite(strat[s].batch_div);
+    for (int l = 0; l < L; l++)
+        ok = ok && pos_finite(layers[l].h) && pos_finite(layers[l].seq) && nonneg_finite(layers[l].heads) &&
+             nonneg_finite(layers[l].c_lin) && nonneg_finite(layers[l].c_attn) && nonneg_finite(layers[l].p_coef) &&
+             nonneg_finite(layers[l].n_ar) && nonneg_finite(layers[l].act_rep) && nonneg_finite(layers[l].act_tp) &&
+             nonneg_finite(layers[l].act_attn);
+    return ok ? 0 : ORC_BAD_INPUT;
+}
+
+/* One instance: every (layer, strategy) and every (s', s). Outputs may be NULL.  Returns 0, or ORC_BAD_INPUT for
+ * a bad descriptor: the integer tables are then filled with -1 (which the search's validation flags in turn)
+ * and the double outputs are left untouched. */
+int orc_eval_costs(int L, int S, const orc_layer *layers, const orc_strategy *strat, const orc_inst *in,
+                   double *time_s, double *mem_bytes, int32_t *time_q, int32_t *mem_q, int32_t *trans_q)
+{
+    if (orc_check_descriptors(L, S, layers, strat, in)) {
+        for (int e = 0; e < L * S; e++) {
+            if (time_q) time_q[e] = -1;
+            if (mem_q) mem_q[e] = -1;
+        }
+        if (trans_q)
+            for (int e = 0; e < S * S; e++) trans_q[e] = -1;
+        return ORC_BAD_INPUT;
+    }
     for (int l = 0; l < L; l++)
         for (int s = 0; s < S; s++) {
             double t, b;
@@ -286,6 +318,7 @@ void orc_eval_costs(int L, int S, const orc_layer *layers, const orc_strategy *s
             for (int c = 0; c < S; c++)
                 trans_q[a * S + c] = orc_quant_time(orc_trans_cost(&layers[0], &strat[a], &strat[c], in),
                                                     in->time_unit_ns);
+    return 0;
 }
 
 /* ------------------------------------------------------------------ outer selection

@@ -125,6 +125,15 @@ def eval_costs(layers, strat, inst, L: int):
     return ts, mb, tq, mq, xq
 
 
+def descriptor_status(layers, strat, inst, L: int) -> int:
+    """0, or BAD_INPUT when a descriptor of the instance (its parameters, the strategy table, its L layers) is one
+    no profiler could have produced (see orc_check_descriptors); eval_costs then fills the integer tables with -1."""
+    layers = np.ascontiguousarray(layers); strat = np.ascontiguousarray(strat)
+    inst = np.ascontiguousarray(inst).reshape(1)
+    vp = lambda a: a.ctypes.data_as(C.c_void_p)
+    return int(lib().orc_check_descriptors(L, len(strat), vp(layers), vp(strat), vp(inst)))
+
+
 def search(time, mem, trans, M: int, budget=None, use_A: bool = False):
     """Whole path for one instance on integer tables: validate, DP, optimum, plan."""
     st = validate(time, mem, trans)

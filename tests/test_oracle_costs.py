@@ -154,3 +154,33 @@ def test_time_grows_with_batch_and_rounding(orc):
     assert [lib.orc_quant_mem(v, 4.0) for v in (0.0, 0.1, 4.0, 4.1, 8.0)] == [0, 1, 1, 2, 2]
     assert lib.orc_quant_time(1e30, 1.0) == 2 ** 30 and lib.orc_quant_mem(1e30, 1.0) == 2 ** 30
     assert lib.orc_quant_time(float("nan"), 1.0) == 2 ** 30
+
+
+def test_descriptors_no_profiler_could_produce(orc):
+    """What makes an instance BAD_INPUT in the cost model, case by case, and what the integer tables then hold."""
+    w = inputs.config3(B=3)
+    L = 6
+    assert orc.descriptor_status(w.layers[0], w.strat, w.inst[0], L) == 0
+    def bad_inst(field, value):
+        inst = w.inst[1].copy(); inst[field] = value
+        return orc.descriptor_status(w.layers[0], w.strat, inst, L)
+    for field in ("b", "act_mult", "flops_rate", "bw_tp", "bw_dp", "bytes_per_elem", "bin_bytes", "time_unit_ns"):
+        for value in (0.0, -1.0, float("nan"), float("inf")):
+            assert bad_inst(field, value) == orc.BAD_INPUT, (field, value)
+    def bad_strat(field, value):
+        st = w.strat.copy(); st[field][5] = value
+        return orc.descriptor_status(w.layers[0], st, w.inst[0], L)
+    for field, value in (("tp", 0), ("dp", -2), ("zero", 4), ("zero", -1), ("ckpt", 2), ("sp", -1), ("batch_div", 0.0), ("batch_div", float("nan"))):
+        assert bad_strat(field, value) == orc.BAD_INPUT, (field, value)
+    def bad_layer(l, field, value):
+        ly = w.layers[0].copy(); ly[field][l] = value
+        return orc.descriptor_status(ly, w.strat, w.inst[0], L)
+    assert bad_layer(2, "h", 0.0) == orc.BAD_INPUT and bad_layer(5, "seq", float("nan")) == orc.BAD_INPUT
+    assert bad_layer(0, "c_attn", -1.0) == orc.BAD_INPUT and bad_layer(3, "act_tp", float("inf")) == orc.BAD_INPUT
+    assert bad_layer(1, "heads", 0.0) == 0 and bad_layer(1, "c_attn", 0.0) == 0      # zero coefficients are fine (an FFN has no attention term)
+    assert bad_layer(6, "h", -5.0) == 0                                               # beyond the instance's layers: not looked at
+    # the tables of a flagged instance: -1 everywhere, so the search's own validation flags it too
+    inst = w.inst[2].copy(); inst["bw_tp"] = 0.0
+    ts, mb, tq, mq, xq = orc.eval_costs(w.layers[0], w.strat, inst, L)
+    assert (tq == -1).all() and (mq == -1).all() and (xq == -1).all()
+    assert orc.validate(tq, mq, xq) == orc.BAD_INPUT
