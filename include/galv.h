@@ -360,6 +360,20 @@ int galv_layer_optima(galv_ctx* ctx, const galv_shape* shape, const int32_t* L, 
 int galv_stage_partition(galv_ctx* ctx, int32_t Lm, int32_t P, const int32_t* range_opt,
                          int32_t* cuts, int32_t* bottleneck, void* stream);
 
+/*
+ * What GALV_SKIP_INFEASIBLE and GALV_SKIP_DOMINATED would leave out of a search, estimated from its inputs (the
+ * paper has no counterpart; the flags never change a result, only the work, and how much depends on the data).
+ * counts int64 [4], device: [0] tiles of the tiled kernel that lie wholly below the previous layer's feasibility
+ * frontier (the running sum of the layers' smallest mem) out of [1] tiles in all, over layers 1 .. L[i]-1 of every
+ * instance: the exact share GALV_SKIP_INFEASIBLE skips; [2] rows of layer 0 that cannot win in layer 1 (they never
+ * fit, or their time exceeds the layer's smallest by more than the largest transition entry) out of [3] rows: an
+ * indication of what GALV_SKIP_DOMINATED finds, which in later layers depends on the tables themselves.
+ * Instances with L[i] outside 1..Lmax are not counted.  Same table arguments as galv_dp_search.
+ */
+int galv_skip_estimate(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,
+                       const int32_t* time_q, const int32_t* mem_q, const int32_t* trans_q,
+                       int64_t* counts, void* stream);
+
 /* Bytes of device arena galv_search_host needs (0 on invalid shape). */
 size_t galv_search_host_arena_bytes(const galv_ctx* ctx, const galv_shape* shape, int with_model);
 

@@ -38,7 +38,7 @@ EXPORTS = ("galv_create", "galv_destroy", "galv_strerror", "galv_last_error", "g
            "galv_dp_search_static", "galv_select_best", "galv_prune_strategies",
            "galv_compact_tables", "galv_expand_plan", "galv_plan_cost", "galv_graph_create", "galv_graph_launch",
            "galv_graph_destroy", "galv_layer_optima", "galv_stage_partition", "galv_add_switch_cost",
-           "galv_switch_decision")
+           "galv_switch_decision", "galv_skip_estimate")
 
 
 class galv_shape(C.Structure):
@@ -90,6 +90,7 @@ def load_library() -> C.CDLL:
     lib.galv_graph_destroy.argtypes = [vp]
     lib.galv_layer_optima.argtypes = [vp, shp] + [vp] * 6
     lib.galv_stage_partition.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, vp, vp]
+    lib.galv_skip_estimate.argtypes = [vp, shp] + [vp] * 6
     lib.galv_search_host_arena_bytes.argtypes = [vp, shp, C.c_int]
     lib.galv_search_host_arena_bytes.restype = sz
     lib.galv_search_host.argtypes = [vp, shp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -210,6 +211,10 @@ class Galv:
     def galv_layer_optima(self, shape, L, Ct, budget, status, opt_l):
         self._check(self.lib.galv_layer_optima(self.h, C.byref(shape), _ptr(L), _ptr(Ct), _ptr(budget), _ptr(status),
                                                _ptr(opt_l), _stream()))
+
+    def galv_skip_estimate(self, shape, L, time_q, mem_q, trans_q, counts):
+        self._check(self.lib.galv_skip_estimate(self.h, C.byref(shape), _ptr(L), _ptr(time_q), _ptr(mem_q), _ptr(trans_q),
+                                                _ptr(counts), _stream()))
 
     def galv_stage_partition(self, Lm, P, range_opt, cuts, bottleneck):
         self._check(self.lib.galv_stage_partition(self.h, Lm, P, _ptr(range_opt), _ptr(cuts), _ptr(bottleneck), _stream()))

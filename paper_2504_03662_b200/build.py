@@ -1,6 +1,8 @@
 """Builds libgalv.so in-tree with nvcc for sm_100a (cross-compiles without a GPU).
 
-    python -m paper_2504_03662_b200.build [--force] [--verbose]
+    python -m paper_2504_03662_b200.build [--force] [--verbose] [--nvtx]
+
+--nvtx compiles NVTX ranges around the three calls of the path into the library (off by default: no dependency).
 """
 from __future__ import annotations
 
@@ -12,7 +14,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgalv.so")
-SOURCES = ["galv_api.cu", "galv_dp.cu", "galv_backtrack.cu", "galv_costs.cu", "galv_probe.cu", "galv_noalloc.cu", "galv_select.cu", "galv_prune.cu", "galv_graph.cu", "galv_stages.cu", "galv_switch.cu", "galv_cluster.cu"]
+SOURCES = ["galv_api.cu", "galv_dp.cu", "galv_backtrack.cu", "galv_costs.cu", "galv_probe.cu", "galv_noalloc.cu", "galv_select.cu", "galv_prune.cu", "galv_graph.cu", "galv_stages.cu", "galv_switch.cu", "galv_cluster.cu", "galv_estimate.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 # The cost model must round every product and sum on its own (no fused multiply-add).
@@ -34,8 +36,8 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
+def build_library(force: bool = False, verbose: bool = False, nvtx: bool = False) -> str:
+    if not force and not nvtx and not _stale():
         return LIB
     nvcc = _nvcc()
     objdir = os.path.join(PKG, "build")
@@ -43,7 +45,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for src in SOURCES:
         obj = os.path.join(objdir, src.replace(".cu", ".o"))
-        cmd = [nvcc, *ARCH, *COMMON, *PER_FILE.get(src, []), *(["-Xptxas", "-v"] if verbose else []),
+        cmd = [nvcc, *ARCH, *COMMON, *PER_FILE.get(src, []), *(["-Xptxas", "-v"] if verbose else []), *(["-DGALV_NVTX"] if nvtx else []),
                "-c", os.path.join(CSRC, src), "-o", obj]
         procs.append((src, obj, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     objs = []
@@ -55,10 +57,10 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
             raise RuntimeError(f"nvcc failed on {src}")
         objs.append(obj)
     tmp = f"{LIB}.{os.getpid()}.tmp"
-    subprocess.check_call([nvcc, *ARCH, "-shared", "-o", tmp, *objs])
+    subprocess.check_call([nvcc, *ARCH, "-shared", "-o", tmp, *objs, *(["-ldl"] if nvtx else [])])
     os.replace(tmp, LIB)
     return LIB
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="--verbose" in sys.argv, nvtx="--nvtx" in sys.argv))

@@ -8,6 +8,20 @@
 
 #include "galv_internal.h"
 
+// Built with -DGALV_NVTX (python -m paper_2504_03662_b200.build --nvtx), the three calls of the path open a named
+// range each, so that a timeline profiler shows cost model / search / plan step; the default build has no such
+// dependency.
+#ifdef GALV_NVTX
+#include <nvtx3/nvToolsExt.h>
+struct GalvRange {
+    explicit GalvRange(const char* name) { nvtxRangePushA(name); }
+    ~GalvRange() { nvtxRangePop(); }
+};
+#define GALV_RANGE(name) GalvRange galv_range_(name)
+#else
+#define GALV_RANGE(name) do { } while (0)
+#endif
+
 namespace {
 
 void set_err(galv_ctx* ctx, const char* fmt, const char* detail = "")
@@ -133,6 +147,7 @@ int galv_eval_costs(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const
                     double* time_s, double* mem_bytes, int32_t* time_q, int32_t* mem_q, int32_t* trans_q,
                     int32_t* status, void* stream)
 {
+    GALV_RANGE("galv_eval_costs");
     if (!ctx) return GALV_ERR_INVALID_ARG;
     if (!shape_ok(sh)) { set_err(ctx, "galv_eval_costs: shape outside limits"); return GALV_ERR_INVALID_ARG; }
     if (!L || !layers || !strat || !inst || !time_q || !mem_q || !trans_q || !status) {
@@ -163,6 +178,7 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const 
                    const int32_t* mem_q, const int32_t* trans_q, int32_t* C, uint8_t* A, int32_t* C_last,
                    void* workspace, size_t workspace_bytes, int32_t* status, void* stream)
 {
+    GALV_RANGE("galv_dp_search");
     if (!ctx) return GALV_ERR_INVALID_ARG;
     if (!shape_ok(sh)) { set_err(ctx, "galv_dp_search: shape outside limits"); return GALV_ERR_INVALID_ARG; }
     if (!L || !time_q || !mem_q || !trans_q || !C_last || !status) {
@@ -227,6 +243,7 @@ int galv_backtrack(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const 
                    const int32_t* C_last, const int32_t* budget, int32_t* opt_cost, int32_t* plan,
                    int32_t* mem_used, int32_t* status, void* stream)
 {
+    GALV_RANGE("galv_backtrack");
     if (!ctx) return GALV_ERR_INVALID_ARG;
     if (!shape_ok(sh)) { set_err(ctx, "galv_backtrack: shape outside limits"); return GALV_ERR_INVALID_ARG; }
     if (!L || !time_q || !mem_q || !trans_q || !C_last || !opt_cost || !status) {
