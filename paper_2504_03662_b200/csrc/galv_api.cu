@@ -213,6 +213,8 @@ int galv_dp_search(galv_ctx* ctx, const galv_shape* sh, const int32_t* L, const 
     a.istart = reinterpret_cast<long long*>(ws + w.istart);
     a.tcount = reinterpret_cast<int32_t*>(ws + w.tcount);
     a.trans_p = reinterpret_cast<uint32_t*>(ws + w.trans_p);
+    a.trans_k = reinterpret_cast<int32_t*>(ws + w.trans_p);
+    a.keyed = 0;
     a.err = reinterpret_cast<int32_t*>(ws + w.err);
     a.tile_done = reinterpret_cast<int32_t*>(ws + w.tile_done);
     a.maxmem = a.err + 1;

@@ -375,6 +375,18 @@ __global__ void pack_trans_kernel(long long n_mats, int S, const int32_t* __rest
     }
 }
 
+// trans_k = trans_q with every entry << 6 when keys are possible (largest entry of the valid instances < 2^24, so that
+// rebased cost + entry, shifted, stays below 2^31), else a plain copy; maxmem[3] tells the layer kernels which.
+__global__ void key_trans_kernel(long long n, const int32_t* __restrict__ trans_q, int32_t* __restrict__ trans_k, int32_t* __restrict__ maxmem)
+{
+    const int sh = maxmem[1] < (1 << 24) ? 6 : 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) maxmem[3] = sh != 0;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+        const int v = trans_q[e];
+        trans_k[e] = v < 0 ? v : (int)((unsigned)v << sh);     // negative entries belong to flagged instances: never read
+    }
+}
+
 // ---------------------------------------------------------------- tiled layer kernel
 //
 // Work items are (layer, instance, m'-tile, s-block), numbered layer by layer.  CTAs take them one
@@ -487,6 +499,10 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
     const int KS = P16 ? S : pl.ks, NKC = P16 ? 1 : pl.nkc, NST = P16 ? 2 : pl.nst;
+    // Argmin table with keys (S <= 64, all rows of a tile in one stage, transition entries below 2^24): the previous-layer
+    // values of a tile are rebased per column and rewritten as (difference << 6 | row), the transition entries come
+    // shifted by 6 bits, and ONE fused add-min per relaxation carries cost and lowest minimising row together.
+    const bool keyed = ARG && !DOM && !P16 && a.keyed && a.maxmem[3] != 0;
     const int Q = S / 2;                                   // packed path: row pairs
     const int l_last = MULTI ? l_last_arg : l_first + 1;  // single-layer instantiation: loops over l run once
     int32_t* const tile_done = MULTI ? a.tile_done : nullptr;
@@ -621,7 +637,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
             const int sb0 = pos.sb * SB;
             const int sbw = min(SB, S - sb0);             // strategies of this block that exist
             const int yc = row0 + i * inst_rows;
-            const int32_t* T = a.trans_q + (size_t)i * a.trans_inst + (size_t)l * a.trans_layer + sb0;
+            const int32_t* T = ((ARG && a.keyed) ? a.trans_k : a.trans_q) + (size_t)i * a.trans_inst + (size_t)l * a.trans_layer + sb0;
             const int yt = a.trans_layer ? (i * a.Lmax + l) * S : i * S;     // row of trans(0, .) in the tensor map
             // a tile wholly below the previous layer's feasibility frontier reads nothing but +inf: no loads
             const bool skip = a.front && m0 + TMB - 1 < a.front[(size_t)i * a.Lmax + (l - 1)];
@@ -1152,6 +1168,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
         }
     }
     const int kmax = (DOM && !P16) ? a.maxmem[1] : 0;      // largest transition entry (read once: a global load inside the loop waits behind the SM's stores)
+    const int kmaxk = keyed ? a.maxmem[1] : 0;
     for (int it = 0;; ++it) {
         int l = 0, mw = 0, nj = 0;
         ItemPos pos = {0, 0, 0};
@@ -1159,10 +1176,12 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
         for (int j = 0; j < TM; ++j)
 #pragma unroll
             for (int u = 0; u < TS; ++u) {
-                acc[j][u] = kInf;                            // min over candidates never exceeds kInf
+                acc[j][u] = keyed ? 0x7fffffff : kInf;       // min over candidates never exceeds kInf (keys: the largest key)
                 if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = 255;
             }
         int mm[TS], tt[TS], inst = 0;
+        int kbase[ARG ? TM : 1];                             // keyed argmin: the smallest previous-layer value of each of this lane's columns
+        (void)kbase;
         for (int kc = 0; kc < NKC; ++kc, ++n) {
             const int st = cst;                             // = n % NST, phase cph = (n / NST) & 1
             if (!mbar_wait(&full_bar[st], cph)) {
@@ -1196,7 +1215,84 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
             // this warp's columns inside their box, and its 8 trans columns
             const int32_t* cs = stage0 + st * stage_elems + ((ms * (32 * TM)) / BOXC) * (KS * BOXC) + (ms * (32 * TM)) % BOXC + lane;
             const int32_t* ts = stage0 + st * stage_elems + KS * TMB + sg * TS;
-            if constexpr (DOM && !P16) {
+            bool keyed_done = false;
+            if constexpr (ARG && !DOM && !P16) {
+                if (keyed) {
+                    keyed_done = true;
+                    // column minima of this warp's own columns over every row (each warp of the group scans them for itself:
+                    // there is no room for a shared array of them beside the stages)
+#pragma unroll
+                    for (int j = 0; j < TM; ++j) kbase[ARG ? j : 0] = kInf;
+                    for (int r = 0; r < kn; ++r)
+#pragma unroll
+                        for (int j = 0; j < TM; ++j) kbase[ARG ? j : 0] = min(kbase[ARG ? j : 0], cs[r * BOXC + j * 32]);
+                    // every warp of the group has read the raw values before any of them is overwritten
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&conv_bar[ms]);
+                    if (!mbar_wait(&conv_bar[ms], 0)) {                     // two phases of this barrier per item: scan done, keys written
+                        if (lane == 0) atomicExch(a.err, 1);
+                        return;
+                    }
+                    if (kn > 0) {
+                        // this warp's share of the rows, all columns of the group: value -> key.  A candidate more than the
+                        // largest transition entry above its column's best cannot win or tie, so the difference is capped there.
+                        const int K = kmaxk + 1;
+                        int32_t* const cw = const_cast<int32_t*>(cs);
+                        const int RW = (kn + NSG - 1) / NSG;
+                        for (int r = sg * RW; r < min(kn, sg * RW + RW); ++r)
+#pragma unroll
+                            for (int j = 0; j < TM; ++j) {
+                                const int d = __viaddmin_s32(cw[r * BOXC + j * 32], -kbase[ARG ? j : 0], K);
+                                cw[r * BOXC + j * 32] = d * 64 + r;
+                            }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&conv_bar[ms]);
+                    if (!mbar_wait(&conv_bar[ms], 1)) {
+                        if (lane == 0) atomicExch(a.err, 1);
+                        return;
+                    }
+                    if (nj > 0) {
+                        int k = 0;
+                        auto ksteps = [&](auto ku) {
+                            constexpr int K = decltype(ku)::value;
+                            for (; k + K <= kn; k += K) {
+#pragma unroll
+                                for (int kk = 0; kk < K; ++kk) {
+                                    int c[TM];
+#pragma unroll
+                                    for (int j = 0; j < TM; ++j) c[j] = cs[kk * BOXC + j * 32];
+                                    const int4 t0 = *reinterpret_cast<const int4*>(ts + kk * SB);
+                                    const int4 t1 = *reinterpret_cast<const int4*>(ts + kk * SB + 4);
+                                    const int t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+                                    for (int j = 0; j < TM; ++j)
+#pragma unroll
+                                        for (int u = 0; u < TS; ++u) acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
+                                }
+                                cs += K * BOXC;
+                                ts += K * SB;
+                            }
+                        };
+                        ksteps(std::integral_constant<int, 16>());
+                        ksteps(std::integral_constant<int, 4>());
+                        ksteps(std::integral_constant<int, 1>());
+                        // key -> (cost before time(l,s), row): what the epilogue expects of the plain loop
+#pragma unroll
+                        for (int j = 0; j < TM; ++j)
+#pragma unroll
+                            for (int u = 0; u < TS; ++u) {
+                                const int key = acc[j][u];
+                                arg[ARG ? j : 0][ARG ? u : 0] = key & 63;
+                                acc[j][u] = kbase[ARG ? j : 0] >= kInf ? kInf : kbase[ARG ? j : 0] + (key >> 6);
+                            }
+                    }
+                    // the stage was rewritten by plain stores; the next load into it comes through the async proxy
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+            }
+            if (keyed_done) {
+            } else if constexpr (DOM && !P16) {
                 // Dominated rows left out (one chunk per item, S <= 64: the host takes this instantiation only then).
                 // A candidate more than the largest transition entry above its column's best cannot win or tie;
                 // a row that is such in every column of this group's tile is not relaxed.  Each warp scans its
@@ -1473,7 +1569,7 @@ WsLayout galv_ws_layout(const galv_shape* sh)
     w.order = off;   off = align256(off + (size_t)sh->B * 4);
     w.nactive = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.scratch = off; off = align256(off + (size_t)4 * (sh->Lmax + 2) * 4);    // two int32 arrays, one 64-bit array
-    w.err = off;     off = align256(off + 16);                 // error flag, largest mem, largest trans, path chosen
+    w.err = off;     off = align256(off + 32);                 // error flag, largest mem, largest trans, path chosen, keyed argmin
     w.minmem_l = off; off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.ntiles = off;   off = align256(off + (size_t)(sh->Lmax + 1) * 4);
     w.istart = off;   off = align256(off + (size_t)(sh->Lmax + 1) * 8);
@@ -1483,6 +1579,8 @@ WsLayout galv_ws_layout(const galv_shape* sh)
     w.trans_p = off;                                           // packed trans rows for the 16-bit path (S <= 64, S % 4 == 0)
     if (sh->S <= 64 && sh->S % 4 == 0 && !(sh->flags & (GALV_KERNEL_NO_PACKED | GALV_STORE_ARGMIN | GALV_KERNEL_PER_LAYER | GALV_KERNEL_REFERENCE)))
         off = align256(off + (size_t)sh->B * ((sh->flags & GALV_TRANS_PER_LAYER) ? sh->Lmax : 1) * (sh->S / 2) * sh->S * 4);
+    else if (sh->S <= 64 && (sh->flags & GALV_STORE_ARGMIN) && !(sh->flags & GALV_KERNEL_REFERENCE))
+        off = align256(off + (size_t)sh->B * ((sh->flags & GALV_TRANS_PER_LAYER) ? sh->Lmax : 1) * sh->S * sh->S * 4);   // shifted copy for the keyed argmin loop
     w.roll = off;
     if (!(sh->flags & GALV_STORE_C_FULL)) off = align256(off + (size_t)2 * sh->B * sh->S * sh->m_pitch * 4);
     w.total = off;
@@ -1592,7 +1690,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     }
     e = cudaMemsetAsync(a.scratch, 0, (size_t)4 * (Lmax + 2) * 4, st);      // histogram, fill and work counters
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(a.err, 0, 16, st);
+    e = cudaMemsetAsync(a.err, 0, 32, st);                       // error flag, largest mem, largest trans, path, keyed
     if (e != cudaSuccess) return e;
     const bool reference = (sh->flags & GALV_KERNEL_REFERENCE) != 0;
     DpPlan pl;
@@ -1632,13 +1730,23 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
 
     CUtensorMap maps[4];
     std::memset(maps, 0, sizeof(maps));
+    bool keyed_possible = false;
     if (!reference) {
         // previous-layer values as a 2-D tensor [rows of m_pitch columns]; box = ks rows x (<=256) columns
         const int boxc = 32 * pl.tm * ((pl.nms % 2 == 0 && 64 * pl.tm <= 256) ? 2 : 1);
         const size_t rows = a.C ? (size_t)B * Lmax * S : (size_t)2 * B * S;
         if ((e = encode_2d(&maps[0], a.C ? (void*)a.C : (void*)a.roll, (size_t)a.m_pitch, rows, boxc, pl.ks)) != cudaSuccess) return e;
+        // argmin table with keys: the layer kernels read the shifted copy of the transition matrices
+        // (not with GALV_SKIP_DOMINATED: that instantiation walks the live rows with the plain loop)
+        keyed_possible = a.A != nullptr && S <= 64 && pl.nkc == 1 && pl.nsb == 1 && !(sh->flags & GALV_SKIP_DOMINATED);
+        if (keyed_possible) {
+            const long long n = (long long)B * (a.trans_layer ? Lmax : 1) * S * S;
+            long long blocks = (n + 255) / 256;
+            if (blocks > 148 * 8) blocks = 148 * 8;
+            key_trans_kernel<<<(int)blocks, 256, 0, st>>>(n, a.trans_q, a.trans_k, a.err + 1);
+        }
         if (pl.tma_t &&
-            (e = encode_2d(&maps[1], (void*)a.trans_q, (size_t)S, (size_t)B * (a.trans_layer ? Lmax : 1) * S, pl.sb, pl.ks)) != cudaSuccess) return e;
+            (e = encode_2d(&maps[1], keyed_possible ? (void*)a.trans_k : (void*)a.trans_q, (size_t)S, (size_t)B * (a.trans_layer ? Lmax : 1) * S, pl.sb, pl.ks)) != cudaSuccess) return e;
         if (will_p16) {
             // whole tiles (all S rows) of the previous layer; packed trans rows [S/2 row pairs][S]
             const long long n_mats = (long long)B * (a.trans_layer ? Lmax : 1);
@@ -1652,6 +1760,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     DpArgs ap = a;
     ap.withhold = (sh->flags & GALV_DEBUG_WITHHOLD_LOAD) != 0;
     ap.skip_dom = (sh->flags & GALV_SKIP_DOMINATED) != 0;
+    ap.keyed = keyed_possible;
     if (!(sh->flags & GALV_SKIP_INFEASIBLE)) ap.front = nullptr;
     ap.tile_done = nullptr;
     ap.maxmem = a.err + 1;

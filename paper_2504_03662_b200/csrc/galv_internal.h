@@ -57,8 +57,12 @@ struct DpArgs {
     long long* istart;   // [Lmax+1] items of the layers before l (layer 1 starts at 0); [Lmax] = all items
     int32_t* err;        // device error flag
     int32_t* tile_done;  // [B][ntiles_m] finished items per (instance, tile); NULL when layers are separate launches
-    int32_t* maxmem;     // largest mem over the valid instances (min(.., M+1)); [1] largest trans entry; [2] 1: packed 16-bit path
+    int32_t* maxmem;     // largest mem over the valid instances (min(.., M+1)); [1] largest trans entry; [2] 1: packed 16-bit path;
+                         // [3] 1: trans_k holds shifted entries (keyed argmin loop)
     uint32_t* trans_p;   // packed pairs of trans rows for the 16-bit path: [B][(Lmax)][S/2][S], entry = T[2q][s] | T[2q+1][s] << 16
+    int32_t* trans_k;    // argmin table with keys: copy of trans_q with every entry << 6 (same place in the workspace as trans_p;
+                         // a plain copy when the entries are too large for keys: maxmem[3] says which)
+    int keyed;           // the shape allows the keyed argmin loop (S <= 64, all rows of a tile in one stage)
     int32_t* minmem_l;   // [Lmax+1] smallest mem of each layer over the valid instances
     int32_t* front;      // [B][Lmax] feasibility frontier (sum of the layers' smallest mem), or NULL when tiles are never skipped
     int32_t* ntiles;     // [Lmax+1] tiles per instance that can store anything in layer l

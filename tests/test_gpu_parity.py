@@ -777,3 +777,23 @@ def test_cluster_kernel_is_chosen_for_small_batches_only(galv):
     sb = SearchBuffers(galv, inputs.config0(), gb.STORE_C_FULL | gb.STORE_ARGMIN | gb.KERNEL_CLUSTER)
     sb.dp_search()
     assert galv.galv_dp_search_path(sb.shape, sb.workspace) == gb.PATH_TILED_32
+
+
+@pytest.mark.parametrize("S,M,trans_hi,kw", [
+    (64, 1500, 3000, {}), (48, 900, 50000, dict(ragged=True)), (13, 300, 2000, dict(ragged=True)),      # S % 4 != 0: trans rows staged by plain copies
+    (33, 1000, 2, dict(dup_cols=True, time_hi=5)),                                                        # ties everywhere: the lowest row must win
+    (24, 2881, (1 << 24) - 1, dict(time_hi=1000)), (24, 700, 1 << 24, dict(time_hi=1000)),                # the largest entry keys allow; one beyond: plain loop
+    (64, 767, 40, dict(mem_lo=0, mem_hi=0)), (8, 5000, 700, dict(mem_hi=6000)), (1, 100, 5, {}), (40, 513, 100, dict(mem_lo=600, mem_hi=700))])
+def test_argmin_table_with_keys(orc, galv, S, M, trans_hi, kw):
+    """The argmin-table mode with one fused add-min per relaxation on keys (rebased cost << 6 | row): A and C against the
+    oracle where keys apply (S <= 64, entries below 2^24) and where the plain compare-and-select loop takes over; with
+    rows and columns that are +inf, with nothing feasible, and with tiles skipped below the feasibility frontier."""
+    from paper_2504_03662_b200 import binding as gb
+    B, Lmax = 4, 6
+    w = inputs.random_tables(31000 + S + trans_hi % 1000, B, Lmax, S, M, trans_hi=trans_hi, **{**dict(mem_lo=0, mem_hi=max(1, M // 4)), **kw})
+    if S > 1:
+        w.trans_q[0, 0, 1] = trans_hi                            # the largest entry is really there
+        w.mem_q[1, 2, : S // 2] = M + 3                          # +inf rows
+    w.time_q[2, 1, :] = 9                                        # a layer without spread
+    for flags in (gb.STORE_C_FULL | gb.STORE_ARGMIN, gb.STORE_ARGMIN, gb.STORE_C_FULL | gb.STORE_ARGMIN | gb.SKIP_INFEASIBLE):
+        check_batch(orc, galv, w, flags)
