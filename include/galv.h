@@ -165,7 +165,8 @@ size_t galv_dp_workspace_bytes(const galv_ctx* ctx, const galv_shape* shape);
  * tables are left untouched) and never cause an out-of-range access.
  *
  * C       [B][Lmax][S][m_pitch] iff GALV_STORE_C_FULL, else NULL
- * A       same dims, uint8, iff GALV_STORE_ARGMIN, else NULL
+ * A       same dims, uint8, iff GALV_STORE_ARGMIN, else NULL (with S <= 64 and transition entries below 2^24 the
+ *         argmin loop runs one fused add-min per relaxation on keys, rebased cost << 6 | row; same table)
  * C_last  [B][S][m_pitch], always written: layer L[i]-1 of instance i
  * Pad columns M < m < m_pitch are written as GALV_INF / 255.
  * workspace: 256-byte aligned, at least galv_dp_workspace_bytes(shape) bytes,
@@ -213,8 +214,9 @@ int galv_dp_search_path(galv_ctx* ctx, const galv_shape* shape, const void* work
  * columns); B*S*S*2 bytes of packed transition rows when the packed 16-bit
  * loop may run (S <= 64, S % 4 == 0, neither GALV_KERNEL_NO_PACKED nor
  * GALV_STORE_ARGMIN nor GALV_KERNEL_PER_LAYER; times Lmax with
- * GALV_TRANS_PER_LAYER); and 2*B*S*m_pitch*4 bytes when the full table is not
- * kept.  So batches of a few hundred instances with the full table fit; large
+ * GALV_TRANS_PER_LAYER), or B*S*S*4 bytes of shifted transition entries with
+ * GALV_STORE_ARGMIN and S <= 64 (the argmin loop on keys); and 2*B*S*m_pitch*4
+ * bytes when the full table is not kept.  So batches of a few hundred instances with the full table fit; large
  * batches fit only with GALV_KERNEL_NO_PACKED (B = 1024, S = 32 needs 2 MiB
  * for the packed rows alone), and the rolling two-layer mode only for small
  * B*S*m_pitch.  Ask galv_dp_workspace_bytes.  The call itself allocates
