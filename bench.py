@@ -89,10 +89,25 @@ def spawn_ranks(n: int) -> int:
 
 # ------------------------------------------------------------------ CPU oracle legs
 
-def oracle_sample(w, max_layers: int, threads: int):
-    """First `threads` instances, first `max_layers` layers each: integer tables from the oracle's cost model."""
+ORACLE_RELAX_PER_S_PER_THREAD = 1.3e9          # what the plain C oracle does on one host core (measured on the GPU machine's hosts)
+
+
+def oracle_sample_size(w, threads: int, seconds: float):
+    """(instances, layers) of a sample of the workload that keeps `threads` oracle threads busy for about `seconds`."""
+    per_layer = (w.M + 1) * w.S * w.S
+    budget = seconds * ORACLE_RELAX_PER_S_PER_THREAD               # relaxations per thread
+    layers = int(w.Lmax)
+    if per_layer * max(1, layers - 1) > budget:                     # one instance is already too long: fewer layers
+        layers = max(2, int(budget / per_layer) + 1)
+        return min(threads, w.B), layers
+    per_thread = max(1, int(budget / (per_layer * max(1, layers - 1))))
+    return min(w.B, threads * per_thread), layers
+
+
+def oracle_sample(w, max_layers: int, threads: int, instances: int = 0):
+    """First `instances` (default: one per thread) instances, first `max_layers` layers each: integer tables from the oracle's cost model."""
     from oracle import oracle
-    k = min(threads, w.B)
+    k = min(instances or threads, w.B)
     items = []
     for i in range(k):
         Li = min(int(w.L[i]), max_layers)
@@ -127,14 +142,14 @@ def run_reference(args):
     oracle.build()
     w = workload_for(args.workload)
     threads = min(os.cpu_count() or 1, w.B)
-    max_layers = max(2, min(w.Lmax, int(2.5e8 * 3.0 / ((w.M + 1) * w.S * w.S)) + 1))     # ~3 s of work per thread
-    items, cells = oracle_sample(w, max_layers, threads)
+    n_inst, max_layers = oracle_sample_size(w, threads, 4.0)         # ~4 s of work per thread and step
+    items, cells = oracle_sample(w, max_layers, threads, n_inst)
     for _ in range(args.warmup):
         oracle_run(w, items, threads)
     ts = [oracle_run(w, items, threads) for _ in range(args.steps)]
     t = sum(ts) / len(ts)
     value = cells / t
-    sample = f"first {len(items)} instances x first {max_layers} layers per step, one instance per thread"
+    sample = f"first {len(items)} instances x first {max_layers} layers per step, one instance at a time per thread"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -538,12 +553,12 @@ def main():
         from oracle import oracle
         oracle.build()
         threads = min(os.cpu_count() or 1, w.B, 32)
-        max_layers = max(2, min(w.Lmax, int(2.5e8 * 10.0 / ((w.M + 1) * w.S * w.S)) + 1))   # ~10 s of work per thread
-        items, cells = oracle_sample(w, max_layers, threads)
+        n_inst, max_layers = oracle_sample_size(w, threads, 15.0)    # ~15 s of work per thread
+        items, cells = oracle_sample(w, max_layers, threads, n_inst)
         tc = oracle_run(w, items, threads)
         t1 = oracle_run(w, items[:1], 1)                          # the same search on one core
         line["cpu_baseline"] = {"value": cells / tc, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": tc,
-                                "sample": f"first {len(items)} instances x first {max_layers} layers, one instance per thread",
+                                "sample": f"first {len(items)} instances x first {max_layers} layers, one instance at a time per thread",
                                 "single_core_value": cells / len(items) / t1}
     elif rank == 0:
         line["cpu_baseline"] = None
