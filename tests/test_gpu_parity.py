@@ -797,3 +797,52 @@ def test_argmin_table_with_keys(orc, galv, S, M, trans_hi, kw):
     w.time_q[2, 1, :] = 9                                        # a layer without spread
     for flags in (gb.STORE_C_FULL | gb.STORE_ARGMIN, gb.STORE_ARGMIN, gb.STORE_C_FULL | gb.STORE_ARGMIN | gb.SKIP_INFEASIBLE):
         check_batch(orc, galv, w, flags)
+
+
+@pytest.mark.parametrize("block", range(6))
+def test_cluster_kernel_against_reference_kernel_on_many_shapes(galv, block):
+    """Consistency stress of the cluster kernel (column split, pushes that cross one or several CTAs, fills, rounds of
+    clusters, per-layer transition matrices): on random shapes, cluster sizes and memory distributions its tables must
+    equal those of the one-thread-per-cell kernel, which other tests tie to the oracle.  Two runs per shape on the same
+    buffers."""
+    import torch
+    from paper_2504_03662_b200 import binding as gb
+    from paper_2504_03662_b200.search import SearchBuffers
+    rng = np.random.default_rng(4200 + block)
+    ran = 0
+    for case in range(12):
+        S = int(rng.choice([1, 3, 8, 13, 24, 32, 40, 48, 64, 100, 128]))
+        Lmax = int(rng.integers(1, 14))
+        M = int(rng.integers(95, 4000))
+        B = int(rng.choice([1, 2, 5, 16, 40, 130]))
+        mem_hi = int(rng.choice([0, 5, M // 30 + 1, M // 4 + 1, M + 50, 3 * M]))       # up to shifts that skip whole CTAs and never fit
+        w = inputs.random_tables(61000 + 100 * block + case, B, Lmax, S, M, ragged=bool(rng.integers(0, 2)), mem_lo=0, mem_hi=mem_hi,
+                                 trans_hi=int(rng.choice([0, 9, 40000])), time_hi=int(rng.choice([5, 10 ** 4, 10 ** 6])))
+        if Lmax > 2 and rng.integers(0, 2):
+            w.mem_q[:, int(rng.integers(1, Lmax)), :] += M // 2                          # one heavy layer
+        if case % 4 == 3 and Lmax > 1:                                                   # one transition matrix per layer
+            w.trans_q = np.ascontiguousarray(np.repeat(w.trans_q[:, None], Lmax, 1))
+            w.trans_q[:, 1:] += rng.integers(0, 50, size=(B, Lmax - 1, S, S), dtype=np.int32)
+        size = int(rng.choice([0, 0, 1, 2, 3, 4, 6, 8, 11, 16]))
+        flags = gb.STORE_C_FULL | (gb.CLUSTER_SIZE(size) if size else gb.KERNEL_CLUSTER)
+        ref = SearchBuffers(galv, w, gb.STORE_C_FULL | gb.KERNEL_REFERENCE)
+        ref.dp_search(); ref.backtrack()
+        one = SearchBuffers(galv, w, flags)
+        for _ in range(2):
+            one.C.fill_(-7); one.C_last.fill_(-7)
+            one.dp_search(); one.backtrack()
+            torch.cuda.synchronize()
+            if galv.galv_dp_search_path(one.shape, one.workspace) != gb.PATH_CLUSTER:
+                break                                            # this size is not possible for this shape: nothing to compare
+            ran += 1
+            st = ref.status.cpu().numpy()
+            assert (one.status.cpu().numpy() == st).all(), (block, case)
+            assert torch.equal(one.opt_cost, ref.opt_cost) and torch.equal(one.plan, ref.plan), (block, case)
+            for i in np.flatnonzero((st & ~1) == 0):
+                Li = int(w.L[i])
+                assert torch.equal(one.C[i, :Li], ref.C[i, :Li]), (block, case, int(i), S, Lmax, M, B, size)
+            ok = torch.from_numpy((st & ~1) == 0).to(one.C_last.device)
+            assert torch.equal(one.C_last[ok], ref.C_last[ok]), (block, case)
+        del ref, one
+        torch.cuda.empty_cache()
+    assert ran >= 8                                              # most of the shapes did run on the cluster kernel
