@@ -291,6 +291,7 @@ __global__ void __launch_bounds__(416, 1) cluster_search_kernel(const ClArgs a, 
     };
     if (warp == NW && Li > 2) fetch_rows(2, raw_m, raw_t);
     // every CTA of the cluster has started and holds its layer 0 before anyone writes into a neighbour
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");            // layer 0 goes to the table by a bulk store
     cluster_barrier();
 
     for (int l = 1; l < Li; ++l) {
@@ -432,6 +433,9 @@ __global__ void __launch_bounds__(416, 1) cluster_search_kernel(const ClArgs a, 
                 }
             }
         }
+        // What this thread stored into shared memory, its own CTA's or a neighbour's, is read next by the bulk store of
+        // the CTA that owns it (async proxy): the writer orders it for that proxy before the barrier that publishes it.
+        asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");
         cluster_barrier();                                                  // layer l is complete everywhere
     }
 
