@@ -25,6 +25,7 @@
 
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <type_traits>
 
 #include "galv_internal.h"
@@ -513,7 +514,9 @@ cudaError_t launch_any(const ClArgs& a, const ClPlan& p, const CUtensorMap& mc, 
 // Clusters of this plan's size and resources the device can hold at once (asked once per kind of launch).
 int max_active_clusters(const galv_ctx* ctx, const ClPlan& p)
 {
-    static std::map<unsigned long long, int> cache;          // a context belongs to one host thread at a time
+    static std::map<unsigned long long, int> cache;          // shared by all contexts of the process
+    static std::mutex cache_mutex;
+    std::lock_guard<std::mutex> lock(cache_mutex);
     const unsigned long long key = ((unsigned long long)ctx->device << 48) | ((unsigned long long)p.cl << 40) |
                                    ((unsigned long long)p.tm << 36) | ((unsigned long long)p.nw << 28) | (unsigned long long)((p.smem + 1023) / 1024);
     auto it = cache.find(key);
