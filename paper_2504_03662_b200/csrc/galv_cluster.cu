@@ -530,17 +530,22 @@ int max_active_clusters(const galv_ctx* ctx, const ClPlan& p)
     return n;
 }
 
-// Register-tile height for g column groups per CTA: the one that leaves the four schedulers of an SM the least work.
+// Register-tile height for g column groups per CTA: the one that gives the busiest warp the least work (units are
+// dealt out to at most 12 warps), then the busiest scheduler, then the smaller tile (more, smaller units spread the
+// cost of the tiles that straddle two CTAs).  Returns the busiest scheduler's work in units of 8*S*2 cycles.
 int tile_cost(int g, int nsg, int* tm_out)
 {
-    int best_tm = 4, best = 1 << 30;
+    int best_tm = 4, best_warp = 1 << 30, best_sched = 1 << 30;
     for (int tm = 4; tm >= 2; --tm) {
         const int units = (g + tm - 1) / tm * nsg;
-        const int cost = (units + 3) / 4 * tm;
-        if (cost < best) { best = cost; best_tm = tm; }
+        int nw = (units + 3) & ~3;
+        if (nw > 12) nw = 12;
+        const int warp = (units + nw - 1) / nw * tm;
+        const int sched = (units + 3) / 4 * tm;
+        if (warp < best_warp || (warp == best_warp && sched <= best_sched)) { best_warp = warp; best_sched = sched; best_tm = tm; }
     }
     *tm_out = best_tm;
-    return best;
+    return best_sched;
 }
 
 }  // namespace
