@@ -291,6 +291,7 @@ def main():
     ap.add_argument("--no-packed", action="store_true", help="keep the 32-bit inner loop where the packed 16-bit one would run")
     ap.add_argument("--no-cluster", action="store_true", help="keep the tiled kernels where the small-batch cluster kernel would run")
     ap.add_argument("--instance", type=int, default=-1, help="search only this instance of the workload (single re-search latency)")
+    ap.add_argument("--cost-model-only", action="store_true", help="only the bandwidth-sized cost-model pass (profiler captures); prints its figures")
     ap.add_argument("--skip-dominated", action="store_true", help="run with GALV_SKIP_DOMINATED (profiler captures; the roofline keys then do not apply)")
     ap.add_argument("--batch", type=int, default=0, help="trim the workload to its first instances (profiler captures)")
     ap.add_argument("--layers", type=int, default=0, help="trim the workload to its first layers (profiler captures)")
@@ -336,6 +337,16 @@ def main():
     galv = gb.Galv(local)
     for _ in range(8):                                           # bring the clocks up before short workloads are timed
         galv.galv_probe_int_alu(0, 4096)
+    if args.cost_model_only:
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except OSError:
+            pass
+        print(json.dumps({"cost_model_scaled": cost_model_scaled(torch, galv, peaks.get("hbm_gbs", 6650.0), lambda: None),
+                          "hbm_peak": "of measured" if peaks else "of fallback"}))
+        galv.close()
+        return
     w = workload_for(args.workload, rank, args.batch, args.layers)
     if args.instance >= 0:
         w = w.take([args.instance])

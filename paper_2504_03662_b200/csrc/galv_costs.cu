@@ -166,6 +166,8 @@ __global__ void __launch_bounds__(kThreads) cost_kernel(int B, int Lmax, int S, 
         for (int l = tid; l < Li; l += kThreads) vr[l] = vr[vr[l]];
     }
     __syncthreads();
+    for (int l = tid; l < Li; l += kThreads) root[l] = slot[root[l]];       // from here on: the position of layer l's kind in the list
+    __syncthreads();
     const int ndist = s_ndist;
     const bool vec = (S & 3) == 0;
     for (int k0 = 0; k0 < ndist; k0 += KC) {
@@ -181,19 +183,21 @@ __global__ void __launch_bounds__(kThreads) cost_kernel(int B, int Lmax, int S, 
         }
         __syncthreads();
         // every layer whose kind is in this chunk takes its row from the table
-        if (vec) {
-            const int S4 = S >> 2;
-            for (int e = tid; e < Li * S4; e += kThreads) {
-                const int l = e / S4, c = e - l * S4;
-                const int k = slot[root[l]] - k0;
-                if (k < 0 || k >= kn) continue;
-                reinterpret_cast<int4*>(time_q + base + (size_t)l * S)[c] = reinterpret_cast<const int4*>(tabq + k * S)[c];
-                reinterpret_cast<int4*>(mem_q + base + (size_t)l * S)[c] = reinterpret_cast<const int4*>(tabm + k * S)[c];
-            }
+        if (vec && (S >> 2) <= kThreads) {
+            // a thread keeps its 16-byte column of the rows and walks down the layers: no division in the loop
+            const int S4 = S >> 2, rows_per_pass = kThreads / S4;
+            const int c = tid % S4, r0 = tid / S4;
+            if (r0 < rows_per_pass)
+                for (int l = r0; l < Li; l += rows_per_pass) {
+                    const int k = root[l] - k0;
+                    if (k < 0 || k >= kn) continue;
+                    reinterpret_cast<int4*>(time_q + base + (size_t)l * S)[c] = reinterpret_cast<const int4*>(tabq + k * S)[c];
+                    reinterpret_cast<int4*>(mem_q + base + (size_t)l * S)[c] = reinterpret_cast<const int4*>(tabm + k * S)[c];
+                }
         } else {
             for (int e = tid; e < Li * S; e += kThreads) {
                 const int l = e / S, s = e - l * S;
-                const int k = slot[root[l]] - k0;
+                const int k = root[l] - k0;
                 if (k < 0 || k >= kn) continue;
                 time_q[base + e] = tabq[k * S + s];
                 mem_q[base + e] = tabm[k * S + s];
@@ -202,7 +206,7 @@ __global__ void __launch_bounds__(kThreads) cost_kernel(int B, int Lmax, int S, 
         if (want_d)
             for (int e = tid; e < Li * S; e += kThreads) {
                 const int l = e / S, s = e - l * S;
-                const int k = slot[root[l]] - k0;
+                const int k = root[l] - k0;
                 if (k < 0 || k >= kn) continue;
                 if (time_s) time_s[base + e] = tabt[k * S + s];
                 if (mem_bytes) mem_bytes[base + e] = tabb[k * S + s];
