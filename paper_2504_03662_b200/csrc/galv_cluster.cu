@@ -124,8 +124,9 @@ __device__ __forceinline__ int fill_count(bool real, int mem, int M, int W, int 
 
 // One cluster per instance (cluster c takes the c-th longest when `sorted`), CTA `rank` of the cluster owns
 // budget columns rank*W .. rank*W+W-1.  Dynamic shared memory: two buffers [S][W] of table values (previous
-// and next layer, swapping), the transition matrix [S][SP8] (two of them with one matrix per layer), and two
-// rows of per-strategy records.  Warps 0..NW-1 compute: warp w takes work units w, w+NW, ...; a unit is
+// and next layer, swapping), the transition matrix [S][SP8] (two of them with one matrix per layer), the push
+// records of this layer and the next (one per column tile and strategy), the fill counts, and a dump row for the
+// stores of strategies that land nowhere.  Warps 0..NW-1 compute: warp w takes work units w, w+NW, ...; a unit is
 // 32*TM columns x 8 strategies, one fused add-min per relaxation, accumulators in registers.  The last warp
 // is the service warp: it sends the finished layer to the table (one tensor-map store), prepares the next
 // layer's records and, with one matrix per layer, fetches the next matrix.
