@@ -975,6 +975,10 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
         constexpr int LPC = 16;                            // columns a warp handles at a time: two lanes per column,
                                                            // each with half of the rows (S / 2 <= 32 values, in registers)
         const int K = a.maxmem[1] + 1;                     // a candidate this far above the column's best cannot win
+        // The ALU pipe is what limits this loop, the multiply-add pipe idles: the plain adds and shifts of the side
+        // work (pack two values, split a result, put it back on its base) are written as multiply-adds with factors
+        // the compiler cannot see through, so that they leave the ALU pipe to the add-mins.
+        const uint32_t one = (uint32_t)(a.S != 0), two16 = one << 16;
         const int rows = S / 2;                            // S % 4 == 0: whole row pairs per lane
         constexpr bool dom = DOM;                          // leave dominated row pairs out (an instantiation of its own:
                                                            // the extra code costs the plain packed loop 4 %)
@@ -1048,7 +1052,8 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                             if (rows == 32 || 2 * q < rows) {
                                 const uint32_t d0 = (uint32_t)__viaddmin_s32(v[2 * q], -mn, K);
                                 const uint32_t d1 = (uint32_t)__viaddmin_s32(v[2 * q + 1], -mn, K);
-                                const uint32_t pk = __byte_perm(d0, d1, 0x5410);  // d0 | d1 << 16
+                                uint32_t pk;                                      // d0 | d1 << 16
+                                asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(pk) : "r"(d1), "r"(two16), "r"(d0));
                                 out[q * TMB] = pk;
                                 if (track && pk != kk) alive |= 1u << q;
                             }
@@ -1151,9 +1156,11 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                     for (int j = 0; j < TM; ++j)
                         if (j < nj) {
                             const uint32_t x = (uint32_t)acc[j][u];
-                            const int w = (int)__vminu2(x, x >> 16);                // the better of the two row parities (upper half: min with 0)
-                            const int v = __viaddmin_s32(bs[j], w, kInf);          // back on the column's base (+inf stays)
-                            R[j * 32] = __viaddmin_s32(v, tt[u], kInf);
+                            uint32_t hi, v;
+                            asm("mul.hi.u32 %0, %1, %2;" : "=r"(hi) : "r"(x), "r"(two16));     // x >> 16
+                            const uint32_t w = __vminu2(x, hi);                     // the better of the two row parities (upper half: min with 0)
+                            asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(v) : "r"(w), "r"(one), "r"((uint32_t)bs[j]));   // back on the column's base
+                            R[j * 32] = (int)__viaddmin_u32(v, (uint32_t)tt[u], (uint32_t)kInf);   // +inf stays: below 2^32 unsigned
                         }
                 }
                 if (ms == 0) {
