@@ -118,19 +118,23 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, lon
             const int32_t* prev = C + ((size_t)i * Lmax + (l - 1)) * slice + (m - mm);
             const int32_t* T = T0 + (size_t)l * trans_layer;       // paid between layers l-1 and l
             sp = 255;
-            for (int base = 0; base < S; base += 32) {
-                const int k = base + lane;
-                bool hit = false;
-                int c = kInf;
-                if (k < S) {
-                    c = prev[(size_t)k * m_pitch];
-                    hit = (c < kInf) && (c + T[k * S + s] == target);
-                }
+            // every row's candidate is asked for before the first is looked at: one round trip to memory, not one per 32 rows
+            int cv[8], tv[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int k = lane + 32 * j;
+                cv[j] = k < S ? prev[(size_t)k * m_pitch] : kInf;
+                tv[j] = k < S ? T[k * S + s] : 0;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (32 * j >= S) break;
+                const bool hit = (cv[j] < kInf) && (cv[j] + tv[j] == target);
                 const unsigned b = __ballot_sync(0xffffffffu, hit);
                 if (b) {
                     const int src = __ffs(b) - 1;
-                    sp = base + src;
-                    cur = __shfl_sync(0xffffffffu, c, src);
+                    sp = 32 * j + src;
+                    cur = __shfl_sync(0xffffffffu, cv[j], src);
                     break;
                 }
             }
