@@ -455,7 +455,7 @@ constexpr int kDescRing = 16;
 // of a warp group's 128-column tile contributes nothing to that tile.  The packed variant notes the live row
 // pairs while it rebases; the 32-bit variant (all S <= 64 rows in one stage) scans its columns first.  Either
 // way the group ORs its live rows together, meets at a barrier and relaxes only those.  Same results.
-template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false, bool DOM = false>
+template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false, bool DOM = false, bool KEY = false>
 __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
                                                                               const __grid_constant__ CUtensorMap map_t)
@@ -469,7 +469,8 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                                                                                     // column group; a multiple of 4 (the record is read 16 bytes at a time)
     static_assert(META % 4 == 0, "item records are read with 16-byte loads");
     constexpr int RS = TMB + 4;                           // staging row: TMB columns + room for the shift
-    constexpr int KU = ARG ? 4 : 16;                      // k-steps per trip of the inner loop
+    constexpr bool ARGR = ARG && !KEY;                    // the minimising row is carried in registers of its own (not inside a key)
+    constexpr int KU = ARGR ? 4 : 16;                     // k-steps per trip of the inner loop
     constexpr int NSW = P16 ? (DOM ? 4 : 2) : 1;          // store warps: the packed path's items are short enough for one
                                                           // warp's row-by-row issue (about 10k cycles a tile) to hold them up;
                                                           // with dominated rows left out the drain of the staging tile is
@@ -477,6 +478,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
     constexpr int RPW = 64 / NSW;                         // staging rows (of at most 64) per store warp
     static_assert(TMB % BOXC == 0 && BOXC % (32 * TM) == 0, "a warp's columns must sit inside one box");
     static_assert(!(ARG && P16) && (!P16 || MULTI), "the packed path keeps no argmin and runs all layers in one launch");
+    static_assert(!KEY || (ARG && MULTI && !P16 && !DOM), "the keys-only instantiation writes an argmin table, all layers in one launch");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
@@ -494,7 +496,11 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
     __shared__ int drained_b;                              // further store warps -> first: items whose rows they have stored completely (one count each)
 
     // Which of the two one-launch kernels runs is decided on the device (largest transition entry).
-    if (MULTI && (a.maxmem[2] != 0) != P16) return;
+    if (MULTI && !KEY && (a.maxmem[2] != 0) != P16) return;
+    // Argmin table: the keys-only kernel (one launch over all layers) runs when the transition entries are small
+    // enough for keys; the launches per layer that follow it then have nothing left to do.
+    if (KEY && a.maxmem[3] == 0) return;
+    if (ARG && !KEY && a.keyed_multi && a.maxmem[3] != 0) return;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.S, M = a.M, m_pitch = a.m_pitch;
@@ -502,7 +508,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
     // Argmin table with keys (S <= 64, all rows of a tile in one stage, transition entries below 2^24): the previous-layer
     // values of a tile are rebased per column and rewritten as (difference << 6 | row), the transition entries come
     // shifted by 6 bits, and ONE fused add-min per relaxation carries cost and lowest minimising row together.
-    const bool keyed = ARG && !DOM && !P16 && a.keyed && a.maxmem[3] != 0;
+    const bool keyed = KEY || (ARG && !DOM && !P16 && a.keyed && a.maxmem[3] != 0);
     const int Q = S / 2;                                   // packed path: row pairs
     const int l_last = MULTI ? l_last_arg : l_first + 1;  // single-layer instantiation: loops over l run once
     int32_t* const tile_done = MULTI ? a.tile_done : nullptr;
@@ -958,7 +964,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
     // ---------------------------------------------------------------- consumers
     const int sg = warp % NSG, ms = warp / NSG;
     int acc[TM][TS];
-    int arg[ARG ? TM : 1][ARG ? TS : 1];
+    int arg[(ARG && !KEY) ? TM : 1][(ARG && !KEY) ? TS : 1];
     (void)arg;
     int n = 0, cst = 0;
     uint32_t cph = 0;
@@ -1184,7 +1190,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
 #pragma unroll
             for (int u = 0; u < TS; ++u) {
                 acc[j][u] = keyed ? 0x7fffffff : kInf;       // min over candidates never exceeds kInf (keys: the largest key)
-                if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = 255;
+                if (ARGR) arg[ARGR ? j : 0][ARGR ? u : 0] = 255;
             }
         int mm[TS], tt[TS], inst = 0;
         int kbase[ARG ? TM : 1];                             // keyed argmin: the smallest previous-layer value of each of this lane's columns
@@ -1285,12 +1291,14 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                         ksteps(std::integral_constant<int, 4>());
                         ksteps(std::integral_constant<int, 1>());
                         // key -> (cost before time(l,s), row): what the epilogue expects of the plain loop
+                        // (the keys-only instantiation splits them in its epilogue)
+                        if constexpr (!KEY)
 #pragma unroll
                         for (int j = 0; j < TM; ++j)
 #pragma unroll
                             for (int u = 0; u < TS; ++u) {
                                 const int key = acc[j][u];
-                                arg[ARG ? j : 0][ARG ? u : 0] = key & 63;
+                                arg[ARGR ? j : 0][ARGR ? u : 0] = key & 63;
                                 acc[j][u] = kbase[ARG ? j : 0] >= kInf ? kInf : kbase[ARG ? j : 0] + (key >> 6);
                             }
                     }
@@ -1298,7 +1306,8 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
             }
-            if (keyed_done) {
+            if constexpr (KEY) {
+            } else if (keyed_done) {
             } else if constexpr (DOM && !P16) {
                 // Dominated rows left out (one chunk per item, S <= 64: the host takes this instantiation only then).
                 // A candidate more than the largest transition entry above its column's best cannot win or tie;
@@ -1358,7 +1367,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                                 for (int u = 0; u < TS; ++u) {
                                     if (ARG) {                  // rows come in ascending order: the lowest row wins a tie
                                         const int cand = c[j] + t[u];
-                                        if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = r; }
+                                        if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARGR ? j : 0][ARGR ? u : 0] = r; }
                                     } else {
                                         acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
                                     }
@@ -1388,7 +1397,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                                     for (int u = 0; u < TS; ++u) {
                                         if (ARG) {
                                             const int cand = c[j] + t[u];
-                                            if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARG ? j : 0][ARG ? u : 0] = k0 + k + kk; }
+                                            if (cand < acc[j][u]) { acc[j][u] = cand; arg[ARGR ? j : 0][ARGR ? u : 0] = k0 + k + kk; }
                                         } else {
                                             acc[j][u] = __viaddmin_s32(c[j], t[u], acc[j][u]);
                                         }
@@ -1414,7 +1423,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
     #pragma unroll
                                 for (int u = 0; u < TS; ++u) {
                                     const int cand = c + t[u];
-                                    if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARG ? j : 0][ARG ? u : 0] = k0 + k; }
+                                    if (cand < acc[j][u]) { acc[j][u] = cand; if (ARG) arg[ARGR ? j : 0][ARGR ? u : 0] = k0 + k; }
                                 }
                             }
                     }
@@ -1451,7 +1460,17 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                 // finite sums stay below kInf and acc <= kInf, so acc + time cannot wrap
 #pragma unroll
                 for (int j = 0; j < TM; ++j)
-                    if (j < nj) R[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
+                    if (j < nj) {
+                        if constexpr (KEY) {
+                            // key = (difference to the column's smallest value) << 6 | row; a column without a finite
+                            // value has base +inf and stays +inf (base + 2^25 does not wrap)
+                            const int v = __viaddmin_s32(kbase[ARG ? j : 0], acc[j][u] >> 6, kInf);
+                            acc[j][u] = v >= kInf ? 255 : (acc[j][u] & 63);      // what the argmin table gets
+                            R[j * 32] = __viaddmin_s32(v, tt[u], kInf);
+                        } else {
+                            R[j * 32] = __viaddmin_s32(acc[j][u], tt[u], kInf);
+                        }
+                    }
             }
             if (ms == 0) {
                 // lane u posts mem of strategy u: selects and one store (eight divergent stores cost a thousand cycles)
@@ -1470,7 +1489,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                         uint8_t* pa = a.A + ((size_t)inst * a.Lmax + l) * slice + (size_t)(s0 + u) * m_pitch + (size_t)(mm[u] + mw + lane);
 #pragma unroll
                         for (int j = 0; j < TM; ++j)
-                            if (j * 32 <= lim) pa[j * 32] = (uint8_t)(acc[j][u] >= kInf ? 255 : arg[ARG ? j : 0][ARG ? u : 0]);
+                            if (j * 32 <= lim) pa[j * 32] = KEY ? (uint8_t)acc[j][u] : (uint8_t)(acc[j][u] >= kInf ? 255 : arg[ARGR ? j : 0][ARGR ? u : 0]);
                     }
             }
         }
@@ -1514,6 +1533,7 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
     auto kern_packed = layer_tiled_kernel<TM, NSG, NMS, false, true, true>;
     auto kern_packed_dom = layer_tiled_kernel<TM, NSG, NMS, false, true, true, true>;
     auto kern_multi_dom = layer_tiled_kernel<TM, NSG, NMS, false, true, false, true>;
+    auto kern_multi_key = layer_tiled_kernel<TM, NSG, NMS, true, true, false, false, true>;
     if (!maps) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(kern_dom, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
@@ -1521,6 +1541,7 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_packed_dom, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         if (e == cudaSuccess && !ARG) e = cudaFuncSetAttribute(kern_multi_dom, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
+        if (e == cudaSuccess && ARG) e = cudaFuncSetAttribute(kern_multi_key, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem);
         return e;
     }
     if (packed) {
@@ -1530,6 +1551,8 @@ cudaError_t launch_one(const DpArgs& a, const DpPlan& pl, int l_first, int l_las
     }
     if (l_last - l_first > 1) {
         void* args[] = {(void*)&a, (void*)&pl, (void*)&l_first, (void*)&l_last, (void*)&maps[0], (void*)&maps[1]};
+        if (ARG)     // argmin table through keys, all layers in one launch
+            return cudaLaunchCooperativeKernel((const void*)kern_multi_key, dim3(pl.grid), dim3((NSG * NMS + 4) * 32), args, (size_t)pl.smem, st);
         // dominated rows are left out where all S <= 64 rows of a tile sit in one stage
         const bool dom = a.skip_dom && pl.nkc == 1 && a.S <= 64;
         return cudaLaunchCooperativeKernel(dom ? (const void*)kern_multi_dom : (const void*)kern_multi, dim3(pl.grid), dim3((NSG * NMS + 4) * 32), args, (size_t)pl.smem, st);
@@ -1771,13 +1794,28 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     if (!(sh->flags & GALV_SKIP_INFEASIBLE)) ap.front = nullptr;
     ap.tile_done = nullptr;
     ap.maxmem = a.err + 1;
-    if (persistent) {
+    ap.keyed_multi = 0;
+    // Argmin table where keys are possible: one cooperative launch over all layers (it returns at once when the device
+    // finds the transition entries too large for keys), then the launches per layer, which return at once when it ran.
+    const bool key_multi = keyed_possible && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
+    if (persistent || key_multi) {
         ap.tile_done = a.tile_done;
         if ((e = cudaMemsetAsync(a.tile_done, 0, (size_t)B * pl.ntiles_m * 4, st)) != cudaSuccess) return e;
     }
     const int pk = ctx->prof_count % 64;
     if (ctx->profiling) cudaEventRecord(ctx->pev[2 * pk], st);
     bool persistent_ran = false;
+    if (key_multi) {
+        e = launch_tiled<true>(ap, pl, 1, Lmax, st, maps);
+        if (e == cudaSuccess) {
+            ap.keyed_multi = 1;
+        } else if (e == cudaErrorCooperativeLaunchTooLarge) {
+            (void)cudaGetLastError();                        // the grid cannot be co-resident right now: one launch per layer does it all
+        } else {
+            return e;
+        }
+        ap.tile_done = nullptr;
+    }
     if (persistent) {
         // packed kernel first where possible, then the 32-bit one: each returns at once unless it is the one chosen
         e = will_p16 ? launch_tiled<false>(ap, pl, 1, Lmax, st, maps, true) : cudaSuccess;

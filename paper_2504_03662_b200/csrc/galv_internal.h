@@ -62,6 +62,7 @@ struct DpArgs {
     uint32_t* trans_p;   // packed pairs of trans rows for the 16-bit path: [B][(Lmax)][S/2][S], entry = T[2q][s] | T[2q+1][s] << 16
     int32_t* trans_k;    // argmin table with keys: copy of trans_q with every entry << 6 (same place in the workspace as trans_p;
                          // a plain copy when the entries are too large for keys: maxmem[3] says which)
+    int keyed_multi;     // the keys-only argmin kernel has been launched over all layers: launches per layer return when it ran
     int keyed;           // the shape allows the keyed argmin loop (S <= 64, all rows of a tile in one stage)
     int32_t* minmem_l;   // [Lmax+1] smallest mem of each layer over the valid instances
     int32_t* front;      // [B][Lmax] feasibility frontier (sum of the layers' smallest mem), or NULL when tiles are never skipped
