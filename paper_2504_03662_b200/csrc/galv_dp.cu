@@ -1189,7 +1189,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
         for (int j = 0; j < TM; ++j)
 #pragma unroll
             for (int u = 0; u < TS; ++u) {
-                acc[j][u] = keyed ? 0x7fffffff : kInf;       // min over candidates never exceeds kInf (keys: the largest key)
+                if (!KEY) acc[j][u] = keyed ? 0x7fffffff : kInf;       // min over candidates never exceeds kInf (keys: the largest key)
                 if (ARGR) arg[ARGR ? j : 0][ARGR ? u : 0] = 255;
             }
         int mm[TS], tt[TS], inst = 0;
@@ -1232,6 +1232,64 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
             if constexpr (ARG && !DOM && !P16) {
                 if (keyed) {
                     keyed_done = true;
+                    if constexpr (KEY) {
+                        // The group's warps share the scan: each reads its share of the rows once (they stay in registers),
+                        // posts the minima of those rows in its first row, reads everyone's after a barrier, and, after a
+                        // second one (all have read the posted minima), writes its rows back as keys.  Three hand-overs an
+                        // item, but a third of the shared-memory reads of a scan of all rows by every warp.
+                        const int K = kmaxk + 1;
+                        const int RW = (kn + NSG - 1) / NSG;            // <= TS rows a warp: the block holds at most NSG * TS
+                        const int r0 = sg * RW, r1 = min(kn, r0 + RW);
+                        int32_t* const cw = const_cast<int32_t*>(cs);
+                        int v[TS][TM], pm[TM];
+#pragma unroll
+                        for (int j = 0; j < TM; ++j) pm[j] = kInf;
+#pragma unroll
+                        for (int rr = 0; rr < TS; ++rr)
+#pragma unroll
+                            for (int j = 0; j < TM; ++j) {
+                                v[rr][j] = r0 + rr < r1 ? cs[(r0 + rr) * BOXC + j * 32] : kInf;
+                                pm[j] = min(pm[j], v[rr][j]);
+                            }
+                        if (r0 < r1)
+#pragma unroll
+                            for (int j = 0; j < TM; ++j) cw[r0 * BOXC + j * 32] = pm[j];
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&conv_bar[ms]);
+                        if (!mbar_wait(&conv_bar[ms], (3 * it) & 1)) {
+                            if (lane == 0) atomicExch(a.err, 1);
+                            return;
+                        }
+#pragma unroll
+                        for (int j = 0; j < TM; ++j) kbase[ARG ? j : 0] = kInf;
+                        for (int r = 0; r < kn; r += RW)
+#pragma unroll
+                            for (int j = 0; j < TM; ++j) kbase[ARG ? j : 0] = min(kbase[ARG ? j : 0], cs[r * BOXC + j * 32]);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&conv_bar[ms]);
+                        if (!mbar_wait(&conv_bar[ms], (3 * it + 1) & 1)) {
+                            if (lane == 0) atomicExch(a.err, 1);
+                            return;
+                        }
+                        // value -> key.  A candidate more than the largest transition entry above its column's best cannot
+                        // win or tie, so the difference is capped there.
+#pragma unroll
+                        for (int rr = 0; rr < TS; ++rr)
+                            if (r0 + rr < r1)
+#pragma unroll
+                                for (int j = 0; j < TM; ++j)
+                                    cw[(r0 + rr) * BOXC + j * 32] = __viaddmin_s32(v[rr][j], -kbase[ARG ? j : 0], K) * 64 + (r0 + rr);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&conv_bar[ms]);
+                        if (!mbar_wait(&conv_bar[ms], (3 * it + 2) & 1)) {
+                            if (lane == 0) atomicExch(a.err, 1);
+                            return;
+                        }
+#pragma unroll
+                        for (int j = 0; j < TM; ++j)
+#pragma unroll
+                            for (int u = 0; u < TS; ++u) acc[j][u] = 0x7fffffff;
+                    } else {
                     // column minima of this warp's own columns over every row (each warp of the group scans them for itself:
                     // there is no room for a shared array of them beside the stages)
 #pragma unroll
@@ -1264,6 +1322,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                     if (!mbar_wait(&conv_bar[ms], 1)) {
                         if (lane == 0) atomicExch(a.err, 1);
                         return;
+                    }
                     }
                     if (nj > 0) {
                         int k = 0;
