@@ -178,7 +178,9 @@ size_t galv_dp_workspace_bytes(const galv_ctx* ctx, const galv_shape* shape);
  * Without an argmin table all layers run in ONE cooperative launch (its CTAs hand
  * finished tiles to one another through counters in the workspace, with bounded
  * waits; on the rolling buffer a tile also waits for the readers of the cells it
- * overwrites); with an argmin table, or with GALV_KERNEL_PER_LAYER, one launch per layer.
+ * overwrites); so does the argmin table where its loop can work on keys (S <= 64, entries
+ * below 2^24, no GALV_SKIP_DOMINATED).  Otherwise with an argmin table, and with
+ * GALV_KERNEL_PER_LAYER, one launch per layer.
  * Nothing synchronises the host, so the call may be captured in a CUDA graph.
  */
 int galv_dp_search(galv_ctx* ctx, const galv_shape* shape, const int32_t* L,

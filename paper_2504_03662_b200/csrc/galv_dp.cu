@@ -19,8 +19,9 @@
 // cooperative launch: CTAs publish finished tiles in global counters and start a
 // tile of the next layer as soon as the tiles it reads are published (bounded
 // waits); on the two-layer rolling buffer a tile also waits for the readers of the
-// cells it overwrites.  With an argmin table: one launch per layer.  Either way plain
-// stream work, capturable in a CUDA graph.
+// cells it overwrites.  The argmin table is written in such a launch too where its loop
+// can work on keys (see the keys-only instantiation); otherwise one launch per layer.
+// Either way plain stream work, capturable in a CUDA graph.
 
 #include <cuda.h>
 
@@ -1789,7 +1790,8 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
     e = cudaMemsetAsync(a.minmem_l, 0x7f, (size_t)(Lmax + 1) * 4, st);
     if (e != cudaSuccess) return e;
     // All layers in one cooperative launch when the grid's CTAs can be co-resident (they wait on one
-    // another's tiles); with an argmin table, on request, or for the reference kernel: one launch per layer.
+    // another's tiles); with an argmin table whose loop cannot work on keys, on request, or for the reference
+    // kernel: one launch per layer.
     // With the two-layer rolling buffer an item also waits for the readers of the cells it overwrites.
     const bool persistent = !reference && !a.A && Lmax > 2 && !(sh->flags & GALV_KERNEL_PER_LAYER);
     // The packed 16-bit kernel is launched as well when the shape allows it; which of the two runs is decided on
