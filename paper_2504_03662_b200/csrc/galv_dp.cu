@@ -456,6 +456,27 @@ constexpr int kDescRing = 16;
 // of a warp group's 128-column tile contributes nothing to that tile.  The packed variant notes the live row
 // pairs while it rebases; the 32-bit variant (all S <= 64 rows in one stage) scans its columns first.  Either
 // way the group ORs its live rows together, meets at a barrier and relaxes only those.  Same results.
+//
+// Roles of a CTA and what each hand-over is (every wait is bounded; a wait that runs out sets a.err and the role leaves):
+//   producer (warp NC)      takes the next item from the global counter, posts its record in desc[] (desc_count), waits for
+//                           the tiles of layer l-1 it reads (tile_done[], acquire at gpu scope; rolling buffer: also for the
+//                           readers of the cells it overwrites, then deps_ok), waits for the stage (empty_bar[stage], all
+//                           consumer warps) and issues the TMA loads, which complete on full_bar[stage] (1 arrival + bytes).
+//   helper (warp NC+1)      reads the record, writes mem / time of the s-block into the stage's item record, gives
+//                           full_bar[stage] its second arrival; for a first tile writes the cells no tile stores (fill_count).
+//   consumers (0 .. NC-1)   wait full_bar[stage], relax, arrive on empty_bar[stage]; wait until the store warps have read the
+//                           previous item out of the staging tile (out_drained), write this item's outputs there, arrive on
+//                           out_full.  conv_bar[column group]: hand-overs inside a group (rebase, keys, live rows).
+//   store warp (NC+2)       waits out_full, orders the staging writes for the async proxy, issues the bulk stores; once they
+//   (+ NC+4.. when packed)  have READ the staging tile: out_drained.  One launch over all layers: once they are COMPLETE, and
+//                           the helper's fill and the other store warps' rows (drained_b) as well: drained_count.
+//   publisher (NC+3)        one proxy fence and one gpu-scope fence for all items handed over since its last round, then one
+//                           relaxed add per item to tile_done[instance][tile]; published_count keeps the store warp within
+//                           kPublishLag records of it (the records live in a ring).
+//   end                     the producer posts a record with layer -1 and arrives on full_bar; the consumers pass it on through
+//                           out_full; the store warp sets store_exit for the publisher.
+// The roles are kept in one function body on purpose: split into member functions of a context object the same code ran
+// 2.6 % (packed loop) to 30 % (keys loop) slower, so the kernel stays as measured.
 template <int TM, int NSG, int NMS, bool ARG, bool MULTI, bool P16 = false, bool DOM = false, bool KEY = false>
 __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 1) layer_tiled_kernel(const DpArgs a, const DpPlan pl, const int l_first, const int l_last_arg,
                                                                               const __grid_constant__ CUtensorMap map_c,
