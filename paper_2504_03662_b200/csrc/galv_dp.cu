@@ -362,7 +362,9 @@ __global__ void layer_reference_kernel(DpArgs a, int l)
 
 // ---------------------------------------------------------------- packed trans rows (16-bit path)
 
-// trans_p[i][(l)][q][s] = T[2q][s] | T[2q+1][s] << 16 (the low 16 bits of each; used only when they all fit)
+// trans_p[i][(l)][p][s] = T[a][s] | T[a + 2][s] << 16 with a = 4 * (p / 2) + p % 2: packed row p pairs rows a and a + 2,
+// as the rebase does (one lane of a column takes the even rows, one the odd).  The low 16 bits of each entry; used only
+// when they all fit.
 __global__ void pack_trans_kernel(long long n_mats, int S, const int32_t* __restrict__ trans_q, uint32_t* __restrict__ trans_p)
 {
     const long long n = n_mats * (S / 2) * S;
@@ -372,7 +374,8 @@ __global__ void pack_trans_kernel(long long n_mats, int S, const int32_t* __rest
         const int q = (int)(mq % (S / 2));
         const long long mat = mq / (S / 2);
         const int32_t* T = trans_q + mat * S * S;
-        trans_p[e] = ((uint32_t)T[(2 * q) * S + s] & 0xffffu) | ((uint32_t)T[(2 * q + 1) * S + s] << 16);
+        const int ra = 4 * (q >> 1) + (q & 1);
+        trans_p[e] = ((uint32_t)T[ra * S + s] & 0xffffu) | ((uint32_t)T[(ra + 2) * S + s] << 16);
     }
 }
 
@@ -491,6 +494,12 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                                                                                     // column group; a multiple of 4 (the record is read 16 bytes at a time)
     static_assert(META % 4 == 0, "item records are read with 16-byte loads");
     constexpr int RS = TMB + 4;                           // staging row: TMB columns + room for the shift
+    // Packed path: the raw tile comes in boxes of 128 columns with 16 more on the right, and the packed rows are 16
+    // words longer than the tile: row pitches of 16 mod 32 words, so that the two lanes that share a column (one the
+    // even rows, one the odd rows) and the two packed rows they write fall into different banks.  (The wider boxes
+    // read an eighth more of the table: 1 % slower where dominated rows are left out and the table traffic is the bound.)
+    constexpr int CB = 128, PBOX = CB + 16, NRB = TMB / CB, PP = TMB + 16;
+    static_assert(!P16 || TMB % CB == 0, "whole raw boxes");
     constexpr bool ARGR = ARG && !KEY;                    // the minimising row is carried in registers of its own (not inside a key)
     constexpr int KU = ARGR ? 4 : 16;                     // k-steps per trip of the inner loop
     constexpr int NSW = P16 ? (DOM ? 4 : 2) : 1;          // store warps: the packed path's items are short enough for one
@@ -542,12 +551,12 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
     // lowest unfinished item can always run: the waits end.
 
     // stage: NBOX boxes of [KS][BOXC] previous-layer values, then [KS][SB] trans values; 128-byte multiples.
-    // Packed path: the raw tile (NBOX boxes of [S][BOXC]) first, then two stages of [Q][TMB] packed values,
+    // Packed path: the raw tile (NRB boxes of [S][PBOX]) first, then two stages of [Q][PP] packed values,
     // [Q][SB] packed trans entries, [TMB] column bases and one word per consumer warp (row pairs alive in its columns).
     int32_t* const raw0 = reinterpret_cast<int32_t*>(smem_raw);
-    const int raw_elems = P16 ? ((S * TMB + 31) & ~31) : 0;
+    const int raw_elems = P16 ? ((S * PBOX * NRB + 31) & ~31) : 0;
     int32_t* const stage0 = raw0 + raw_elems;
-    const int stage_elems = P16 ? ((Q * TMB + Q * SB + TMB + NC + 31) & ~31) : ((KS * (TMB + SB) + 31) & ~31);
+    const int stage_elems = P16 ? ((Q * PP + Q * SB + TMB + NC + 31) & ~31) : ((KS * (TMB + SB) + 31) & ~31);
     int32_t* const meta0 = stage0 + NST * stage_elems;
     // staging tile [SB][RS] + its header: mem(l,s) per row, instance, last-layer flag
     int32_t* const stg0 = meta0 + ((NST * META + 31) & ~31);
@@ -680,11 +689,11 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                 if (skip) {
                     if (lane == 0) mbar_arrive(&full_bar[st]);
                 } else if (!((a.withhold & 1) && blockIdx.x == 0 && n == 0) && lane == 0) {
-                    mbar_expect_tx(&full_bar[st], (uint32_t)(S * TMB + Q * SB) * 4u);
+                    mbar_expect_tx(&full_bar[st], (uint32_t)(S * PBOX * NRB + Q * SB) * 4u);
 #pragma unroll
-                    for (int bx = 0; bx < NBOX; ++bx)
-                        tma_load_2d(raw0 + bx * S * BOXC, &map_c, m0 + bx * BOXC, yc, &full_bar[st]);
-                    tma_load_2d(stage0 + st * stage_elems + Q * TMB, &map_t, 0,
+                    for (int bx = 0; bx < NRB; ++bx)
+                        tma_load_2d(raw0 + bx * S * PBOX, &map_c, m0 + bx * CB, yc, &full_bar[st]);
+                    tma_load_2d(stage0 + st * stage_elems + Q * PP, &map_t, 0,
                                 (a.trans_layer ? i * a.Lmax + l : i) * Q, &full_bar[st]);
                 }
                 __syncwarp();
@@ -1030,8 +1039,8 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
             const int nj = (mw > M) ? 0 : min(TM, (M - mw) / 32 + 1);
             int32_t* const stg = stage0 + st * stage_elems;
             uint32_t* const pkc = reinterpret_cast<uint32_t*>(stg);
-            const uint32_t* const pkt = reinterpret_cast<const uint32_t*>(stg + Q * TMB);
-            int32_t* const basep = stg + Q * TMB + Q * SB;
+            const uint32_t* const pkt = reinterpret_cast<const uint32_t*>(stg + Q * PP);
+            int32_t* const basep = stg + Q * PP + Q * SB;
             uint32_t* const alivep = reinterpret_cast<uint32_t*>(basep + TMB);
             const int32_t* const meta = meta0 + st * META;
             const bool skipped = meta[2 * SB + 1] != 0;     // nothing but +inf to read: no data was loaded
@@ -1045,20 +1054,20 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                 for (int c0 = sg * CW; c0 < cend; c0 += LPC) {
                     const int cg = c0 + cl;                     // column inside the group
                     const int c = ms * (32 * TM) + min(cg, 32 * TM - 1);
-                    const int32_t* rp = raw0 + (c / BOXC) * (S * BOXC) + (c % BOXC) + h * rows * BOXC;
+                    const int32_t* rp = raw0 + (c / CB) * (S * PBOX) + (c % CB) + h * PBOX;    // rows h, h + 2, h + 4, ...
                     int v[32];
                     int mn = kInf;
                     if (rows == 32) {                           // S = 64: no row guards
 #pragma unroll
                         for (int r = 0; r < 32; r += 2) {
-                            v[r] = rp[r * BOXC];
-                            v[r + 1] = rp[(r + 1) * BOXC];
+                            v[r] = rp[(2 * r) * PBOX];
+                            v[r + 1] = rp[(2 * r + 2) * PBOX];
                             mn = __vimin3_s32(mn, v[r], v[r + 1]);
                         }
                     } else {
 #pragma unroll
                         for (int r = 0; r < 32; ++r) {
-                            v[r] = r < rows ? rp[r * BOXC] : kInf;
+                            v[r] = r < rows ? rp[(2 * r) * PBOX] : kInf;
                             mn = min(mn, v[r]);
                         }
                     }
@@ -1072,7 +1081,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                         if (lane == 0) mbar_arrive(&empty_bar[0]);
                     }
                     if (cg < cend) {
-                        uint32_t* out = pkc + (h * (rows / 2)) * TMB + c;
+                        uint32_t* out = pkc + h * PP + c;           // packed row 2q + h: rows 4q + h and 4q + 2 + h
                         // columns past the budget and columns without a finite value produce nothing
                         const bool track = dom && mn < kInf && mw + (c - ms * (32 * TM)) <= M;
 #pragma unroll
@@ -1082,14 +1091,14 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                                 const uint32_t d1 = (uint32_t)__viaddmin_s32(v[2 * q + 1], -mn, K);
                                 uint32_t pk;                                      // d0 | d1 << 16
                                 asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(pk) : "r"(d1), "r"(two16), "r"(d0));
-                                out[q * TMB] = pk;
-                                if (track && pk != kk) alive |= 1u << q;
+                                out[(2 * q) * PP] = pk;
+                                if (track && pk != kk) alive |= 1u << (2 * q + h);
                             }
                         if (h == 0) basep[c] = mn;
                     }
                 }
                 if (dom) {
-                    alive = __reduce_or_sync(0xffffffffu, alive << (h * (rows / 2)));
+                    alive = __reduce_or_sync(0xffffffffu, alive);
                     if (lane == 0) alivep[ms * NSG + sg] = alive;
                 }
             }
@@ -1117,7 +1126,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                         for (int kk = 0; kk < KQ; ++kk) {
                             uint32_t c[TM];
 #pragma unroll
-                            for (int j = 0; j < TM; ++j) c[j] = pc[kk * TMB + j * 32];
+                            for (int j = 0; j < TM; ++j) c[j] = pc[kk * PP + j * 32];
                             const uint4 t0 = *reinterpret_cast<const uint4*>(pt + kk * SB);
                             const uint4 t1 = *reinterpret_cast<const uint4*>(pt + kk * SB + 4);
                             const uint32_t t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
@@ -1127,7 +1136,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                                 for (int u = 0; u < TS; ++u)
                                     acc[j][u] = (int)__viaddmin_u16x2(c[j], t[u], (uint32_t)acc[j][u]);
                         }
-                        pc += KQ * TMB;
+                        pc += KQ * PP;
                         pt += KQ * SB;
                     }
                 };
@@ -1146,7 +1155,7 @@ __global__ void __launch_bounds__((NSG * NMS + (P16 ? (DOM ? 7 : 5) : 4)) * 32, 
                         live &= live - 1;
                         uint32_t c[TM];
 #pragma unroll
-                        for (int j = 0; j < TM; ++j) c[j] = pc[qq * TMB + j * 32];
+                        for (int j = 0; j < TM; ++j) c[j] = pc[qq * PP + j * 32];
                         const uint4 t0 = *reinterpret_cast<const uint4*>(pt + qq * SB);
                         const uint4 t1 = *reinterpret_cast<const uint4*>(pt + qq * SB + 4);
                         const uint32_t t[TS] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
@@ -1739,8 +1748,8 @@ bool galv_dp_make_plan(const galv_ctx* ctx, const galv_shape* sh, DpPlan* pl)
     // stages of its packed form (row pairs), the packed trans rows and the column bases; no argmin table.
     {
         const int q = S / 2;
-        const int raw = (S * pl->tmb * 4 + 127) & ~127;
-        const int pst = ((q * pl->tmb + q * pl->sb + pl->tmb + pl->nsg * pl->nms) * 4 + 127) & ~127;
+        const int raw = (S * 144 * (pl->tmb / 128) * 4 + 127) & ~127;       // boxes of 128 + 16 columns
+        const int pst = ((q * (pl->tmb + 16) + q * pl->sb + pl->tmb + pl->nsg * pl->nms) * 4 + 127) & ~127;
         const int total = raw + 2 * pst + ((2 * (2 * pl->sb + 4) + 31) & ~31) * 4 + staging;
         pl->p16 = S <= 64 && S % 4 == 0 && pl->nsb == 1 && !(sh->flags & GALV_STORE_ARGMIN) && total <= budget;
         pl->p16_smem = total;
@@ -1862,7 +1871,7 @@ cudaError_t galv_dp_launch(galv_ctx* ctx, const galv_shape* sh, const DpArgs& a,
         if (will_p16) {
             // whole tiles (all S rows) of the previous layer; packed trans rows [S/2 row pairs][S]
             const long long n_mats = (long long)B * (a.trans_layer ? Lmax : 1);
-            if ((e = encode_2d(&maps[2], a.C ? (void*)a.C : (void*)a.roll, (size_t)a.m_pitch, rows, boxc, S)) != cudaSuccess) return e;
+            if ((e = encode_2d(&maps[2], a.C ? (void*)a.C : (void*)a.roll, (size_t)a.m_pitch, rows, 144, S)) != cudaSuccess) return e;
             if ((e = encode_2d(&maps[3], (void*)a.trans_p, (size_t)S, (size_t)n_mats * (S / 2), pl.sb, S / 2)) != cudaSuccess) return e;
             long long blocks = (n_mats * (S / 2) * S + 255) / 256;
             if (blocks > 148 * 8) blocks = 148 * 8;
