@@ -40,7 +40,7 @@ ALU_PEAK_GOPS = 148 * 64 * 1.965
 # DRAM bytes (read + write) per LAYER of the layer_tiled_kernel, from the committed ncu captures under
 # profiles/ (captured on the first layers of the same batch: the kernel's traffic grows in proportion
 # to the layers a launch covers, so a launch over Lmax-1 layers moves (Lmax-1) times this).
-NCU_TRAFFIC_BYTES_PER_LAYER = {"config3_heterogeneous": 532.7e6, "config4_research_sweep": 541.1e6}
+NCU_TRAFFIC_BYTES_PER_LAYER = {"config3_heterogeneous": 533.6e6, "config4_research_sweep": 541.1e6}
 
 
 def workload_for(k: int, rank: int = 0, batch: int = 0, layers: int = 0):
