@@ -293,6 +293,7 @@ def main():
     ap.add_argument("--instance", type=int, default=-1, help="search only this instance of the workload (single re-search latency)")
     ap.add_argument("--cost-model-only", action="store_true", help="only the bandwidth-sized cost-model pass (profiler captures); prints its figures")
     ap.add_argument("--skip-dominated", action="store_true", help="run with GALV_SKIP_DOMINATED (profiler captures; the roofline keys then do not apply)")
+    ap.add_argument("--argmin-table", action="store_true", help="run with GALV_STORE_ARGMIN as well (profiler captures; the roofline keys then do not apply)")
     ap.add_argument("--batch", type=int, default=0, help="trim the workload to its first instances (profiler captures)")
     ap.add_argument("--layers", type=int, default=0, help="trim the workload to its first layers (profiler captures)")
     args = ap.parse_args()
@@ -356,7 +357,7 @@ def main():
     with ClockSampler(uuid) as clk:
         sb, r = bench_workload(torch, galv, w, args.steps, args.warmup, barrier,
                                flags=1 | (gb.KERNEL_NO_PACKED if args.no_packed else 0) | (gb.SKIP_DOMINATED if args.skip_dominated else 0)
-                                     | (gb.KERNEL_NO_CLUSTER if args.no_cluster else 0))
+                                     | (gb.KERNEL_NO_CLUSTER if args.no_cluster else 0) | (gb.STORE_ARGMIN if args.argmin_table else 0))
     t = max_over_ranks(r["seconds"])
     clocks = clk.summary()
     value = world * w.cells * args.steps / t
