@@ -247,13 +247,13 @@ def cost_model_scaled(torch, galv, hbm_gbs, barrier, copies=8192):
 
 
 def launches_per_step(w, cluster: bool = False) -> int:
-    if cluster:                                   # cost + trans kernels, ONE cluster kernel for the whole search, backtrack
-        return (2 if w.has_model else 0) + 1 + 1
-    # cost + trans kernels, validate + schedule + base layer, ONE cooperative launch over all layers,
+    if cluster:                                   # the cost model's kernel, ONE cluster kernel for the whole search, backtrack
+        return (1 if w.has_model else 0) + 1 + 1
+    # the cost model's kernel, validate + schedule + base layer, ONE cooperative launch over all layers,
     # copy-last + finalize, backtrack; where the shape allows the packed 16-bit path, the kernel that packs
     # the trans rows and the launch of the other inner-loop variant (it returns at once) come on top
     packable = w.S <= 64 and w.S % 4 == 0
-    return (2 if w.has_model else 0) + 3 + 1 + 2 + 1 + (2 if packable else 0)
+    return (1 if w.has_model else 0) + 3 + 1 + 2 + 1 + (2 if packable else 0)
 
 
 def bench_workload(torch, galv, w, steps, warmup, barrier, flags=1):

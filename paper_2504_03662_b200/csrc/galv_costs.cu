@@ -106,17 +106,16 @@ __device__ __forceinline__ bool same_bytes(const galv_layer_desc* a, const galv_
 // One CTA per instance.  Dynamic shared memory: root[Lmax] (the layer whose values layer l takes), slot[Lmax]
 // (position of a distinct layer in the list), list[Lmax] (the distinct layers), then the table of one chunk of
 // distinct layers: tq/mq int32 [KC][S] and, when the doubles are asked for, time_s/mem_bytes [KC][S].
-__global__ void __launch_bounds__(kThreads) cost_kernel(int B, int Lmax, int S, int KC, const int32_t* __restrict__ L,
-                                                        const galv_layer_desc* __restrict__ layers, long long layer_stride_B,
-                                                        const galv_strategy_desc* __restrict__ strat,
-                                                        const galv_inst_params* __restrict__ inst, double* __restrict__ time_s,
-                                                        double* __restrict__ mem_bytes, int32_t* __restrict__ time_q,
-                                                        int32_t* __restrict__ mem_q, int32_t* __restrict__ trans_q,
-                                                        int32_t* __restrict__ status)
+__device__ __forceinline__ void cost_body(const int i, unsigned char* smem_raw, int Lmax, int S, int KC, const int32_t* __restrict__ L,
+                                          const galv_layer_desc* __restrict__ layers, long long layer_stride_B,
+                                          const galv_strategy_desc* __restrict__ strat,
+                                          const galv_inst_params* __restrict__ inst, double* __restrict__ time_s,
+                                          double* __restrict__ mem_bytes, int32_t* __restrict__ time_q,
+                                          int32_t* __restrict__ mem_q, int32_t* __restrict__ trans_q,
+                                          int32_t* __restrict__ status)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_bad, s_ndist;
-    const int i = blockIdx.x, tid = threadIdx.x;
+    const int tid = threadIdx.x;
     const int Li = L[i];
     if (Li < 1 || Li > Lmax) {
         if (tid == 0) status[i] = GALV_STATUS_BAD_INPUT;       // nothing is written for this instance
@@ -228,23 +227,25 @@ __device__ __forceinline__ double pair_factor(const galv_strategy_desc& sa, cons
     return (k - 1.0) / k + spterm;
 }
 // Dynamic shared memory: slot[S] (class of each strategy), rep[S] (one strategy per class), tab[ncls * ncls].
-__global__ void __launch_bounds__(kThreads) trans_kernel(int B, int Lmax, int S, const int32_t* __restrict__ L,
-                                                         const galv_layer_desc* __restrict__ layers, long long layer_stride_B,
-                                                         const galv_strategy_desc* __restrict__ strat,
-                                                         const galv_inst_params* __restrict__ inst, const int32_t* __restrict__ status,
-                                                         int32_t* __restrict__ trans_q, int inst_per_cta)
+// status == nullptr: no earlier kernel has checked the descriptors; the CTA applies the cost kernel's own tests and
+// leaves a flagged instance to it (which writes -1 everywhere).
+__device__ __forceinline__ void trans_body(const int cta, unsigned char* smem_raw, int B, int Lmax, int S, const int32_t* __restrict__ L,
+                                           const galv_layer_desc* __restrict__ layers, long long layer_stride_B,
+                                           const galv_strategy_desc* __restrict__ strat,
+                                           const galv_inst_params* __restrict__ inst, const int32_t* __restrict__ status,
+                                           int32_t* __restrict__ trans_q, int inst_per_cta)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ int s_ncls;
+    __shared__ int s_ncls, s_sbad;
     int* const slot = reinterpret_cast<int*>(smem_raw);
     int* const rep = slot + S;
     int32_t* const tab = rep + S;
     const int tid = threadIdx.x;
-    if (tid == 0) s_ncls = 0;
+    if (tid == 0) { s_ncls = 0; s_sbad = 0; }
     __syncthreads();
     // a strategy opens a class when no earlier one agrees with it in tp, sp and batch_div (compared as bits)
     for (int s = tid; s < S; s += kThreads) {
         const galv_strategy_desc me = strat[s];
+        if (!status && !strat_ok(me)) atomicOr(&s_sbad, 1);
         int first = s;
         for (int o = 0; o < s; ++o) {
             const galv_strategy_desc ot = strat[o];
@@ -261,13 +262,19 @@ __global__ void __launch_bounds__(kThreads) trans_kernel(int B, int Lmax, int S,
         if (slot[s] < 0) slot[s] = slot[-slot[s] - 1];                    // the others copy it (an opener's entry is final by now)
     const bool vec = (S & 3) == 0;
     for (int n = 0; n < inst_per_cta; ++n) {
-        const int i = blockIdx.x * inst_per_cta + n;
+        const int i = cta * inst_per_cta + n;
         if (i >= B) break;
         __syncthreads();                                        // classes known; the last instance's table is no longer read
         const int Li = L[i];
-        if (Li < 1 || Li > Lmax || status[i] != 0) continue;   // out of range: nothing written; bad descriptor: already -1
+        if (Li < 1 || Li > Lmax) continue;                      // out of range: nothing written
+        if (status && status[i] != 0) continue;                 // bad descriptor: already -1
         const galv_layer_desc ly = layers[(long long)i * layer_stride_B];
         const galv_inst_params in = inst[i];
+        if (!status) {
+            int bad = s_sbad | (inst_ok(in) ? 0 : 1);
+            for (int l = tid; l < Li; l += kThreads) bad |= layer_ok(layers[(long long)i * layer_stride_B + l]) ? 0 : 1;
+            if (__syncthreads_or(bad)) continue;                // flagged: the cost role writes -1 into this matrix too
+        }
         for (int e = tid; e < ncls * ncls; e += kThreads) {
             const int ka = e / ncls, kc = e - ka * ncls;
             const galv_strategy_desc sa = strat[rep[ka]], sc = strat[rep[kc]];
@@ -291,6 +298,47 @@ __global__ void __launch_bounds__(kThreads) trans_kernel(int B, int Lmax, int S,
             }
         }
     }
+}
+
+__global__ void __launch_bounds__(kThreads) trans_kernel(int B, int Lmax, int S, const int32_t* __restrict__ L,
+                                                         const galv_layer_desc* __restrict__ layers, long long layer_stride_B,
+                                                         const galv_strategy_desc* __restrict__ strat,
+                                                         const galv_inst_params* __restrict__ inst, const int32_t* __restrict__ status,
+                                                         int32_t* __restrict__ trans_q, int inst_per_cta)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    trans_body(blockIdx.x, smem_raw, B, Lmax, S, L, layers, layer_stride_B, strat, inst, status, trans_q, inst_per_cta);
+}
+
+__global__ void __launch_bounds__(kThreads) cost_kernel(int Lmax, int S, int KC, const int32_t* __restrict__ L,
+                                                        const galv_layer_desc* __restrict__ layers, long long layer_stride_B,
+                                                        const galv_strategy_desc* __restrict__ strat,
+                                                        const galv_inst_params* __restrict__ inst, double* __restrict__ time_s,
+                                                        double* __restrict__ mem_bytes, int32_t* __restrict__ time_q,
+                                                        int32_t* __restrict__ mem_q, int32_t* __restrict__ trans_q,
+                                                        int32_t* __restrict__ status)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    cost_body(blockIdx.x, smem_raw, Lmax, S, KC, L, layers, layer_stride_B, strat, inst, time_s, mem_bytes, time_q, mem_q, trans_q, status);
+}
+
+// The whole cost model in one launch, for batches small enough that a launch counts: the first CTAs write the
+// transition matrices (they run longest and check the descriptors for themselves), the others evaluate one
+// instance's layers each.  Bandwidth-sized batches take the two kernels one after the other (2 % faster there).
+__global__ void __launch_bounds__(kThreads) cost_trans_kernel(int B, int Lmax, int S, int KC, const int32_t* __restrict__ L,
+                                                              const galv_layer_desc* __restrict__ layers, long long layer_stride_B,
+                                                              const galv_strategy_desc* __restrict__ strat,
+                                                              const galv_inst_params* __restrict__ inst, double* __restrict__ time_s,
+                                                              double* __restrict__ mem_bytes, int32_t* __restrict__ time_q,
+                                                              int32_t* __restrict__ mem_q, int32_t* __restrict__ trans_q,
+                                                              int32_t* __restrict__ status, int inst_per_cta)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tblocks = (int)gridDim.x - B;                      // the transition role first: its CTAs run longest
+    if ((int)blockIdx.x >= tblocks)
+        cost_body(blockIdx.x - tblocks, smem_raw, Lmax, S, KC, L, layers, layer_stride_B, strat, inst, time_s, mem_bytes, time_q, mem_q, trans_q, status);
+    else
+        trans_body(blockIdx.x, smem_raw, B, Lmax, S, L, layers, layer_stride_B, strat, inst, nullptr, trans_q, inst_per_cta);
 }
 
 // Stacks too long for the per-instance index arrays in shared memory: descriptors checked by one CTA per
@@ -356,52 +404,62 @@ cudaError_t galv_costs_launch(const galv_shape* sh, const int32_t* L, const galv
 {
     const int S = sh->S, Lmax = sh->Lmax;
     const bool want_d = time_s != nullptr || mem_bytes != nullptr;
+    // instances per CTA of the transition role: the pair-factor table is worth sharing only when CTAs are plenty
+    int ipc = sh->B / (2 * 148);
+    ipc = ipc < 1 ? 1 : (ipc > 8 ? 8 : ipc);
+    const int tblocks = (sh->B + ipc - 1) / ipc;
+    const size_t tsmem = ((size_t)2 * S + (size_t)S * S) * 4;          // at most S classes
     // distinct layers evaluated per pass: as many as fit beside the layer index arrays in 40 KB
     const size_t fixed = (size_t)(3 * Lmax + 4) * 4;
     const size_t per_kind = (size_t)S * (want_d ? 24 : 8);
     const size_t budget = 40 * 1024;
     if (fixed + per_kind + 16 > 200 * 1024) {
-        // very long stacks: no room for the layer index arrays; descriptors checked first, then one thread per element
+        // very long stacks: no room for the layer index arrays; descriptors checked first, then one thread per element,
+        // then the transition matrices of the instances that passed
         check_kernel<<<sh->B, kThreads, 0, st>>>(Lmax, S, L, layers, (long long)layer_stride_B, strat, inst, time_q, mem_q, trans_q, status);
         const long long n = (long long)sh->B * Lmax * S;
         long long blocks = (n + 255) / 256;
         if (blocks > 148 * 16) blocks = 148 * 16;
         cost_direct_kernel<<<(int)blocks, 256, 0, st>>>(sh->B, Lmax, S, L, layers, (long long)layer_stride_B, strat, inst, status, time_s, mem_bytes,
                                                         time_q, mem_q);
-    } else {
-        size_t smem;
-        int kc;
-        if (fixed + per_kind + 16 > budget) {
-            // long stacks: the index arrays alone pass 40 KB; one distinct layer per pass in opted-in shared memory
-            kc = 1;
-            smem = fixed + per_kind + 16;
-            static bool opted = false;
-            if (!opted) {
-                cudaError_t e = cudaFuncSetAttribute(cost_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-                if (e != cudaSuccess) return e;
-                opted = true;
-            }
-        } else {
-            kc = (int)((budget - fixed - 16) / per_kind);
-            if (kc > Lmax) kc = Lmax;
-            smem = fixed + (size_t)kc * per_kind + 16;
-        }
-        cost_kernel<<<sh->B, kThreads, smem, st>>>(sh->B, Lmax, S, kc, L, layers, (long long)layer_stride_B, strat, inst, time_s, mem_bytes,
-                                                   time_q, mem_q, trans_q, status);
-    }
-    // instances per CTA of the transition kernel: the pair-factor table is worth sharing only when CTAs are plenty
-    int ipc = sh->B / (2 * 148);
-    ipc = ipc < 1 ? 1 : (ipc > 8 ? 8 : ipc);
-    const int tblocks = (sh->B + ipc - 1) / ipc;
-    const size_t tsmem = ((size_t)2 * S + (size_t)S * S) * 4;          // at most S classes
-    if (tsmem > 48 * 1024) {
-        static bool opted_t = false;
-        if (!opted_t) {
-            cudaError_t e = cudaFuncSetAttribute(trans_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (2 * 256 + 256 * 256) * 4);
+        if (tsmem > 48 * 1024) {                                   // long stacks or many strategies only; per device, so asked every time
+            cudaError_t e = cudaFuncSetAttribute(trans_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tsmem);
             if (e != cudaSuccess) return e;
-            opted_t = true;
         }
+        trans_kernel<<<tblocks, kThreads, tsmem, st>>>(sh->B, Lmax, S, L, layers, (long long)layer_stride_B, strat, inst, status, trans_q, ipc);
+        return cudaGetLastError();
     }
-    trans_kernel<<<tblocks, kThreads, tsmem, st>>>(sh->B, Lmax, S, L, layers, (long long)layer_stride_B, strat, inst, status, trans_q, ipc);
+    size_t smem;
+    int kc;
+    if (fixed + per_kind + 16 > budget) {
+        // long stacks: the index arrays alone pass 40 KB; one distinct layer per pass
+        kc = 1;
+        smem = fixed + per_kind + 16;
+    } else {
+        kc = (int)((budget - fixed - 16) / per_kind);
+        if (kc > Lmax) kc = Lmax;
+        smem = fixed + (size_t)kc * per_kind + 16;
+    }
+    if (sh->B > 1024) {
+        if (smem > 48 * 1024) {                                   // long stacks or many strategies only; per device, so asked every time
+            cudaError_t e = cudaFuncSetAttribute(cost_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        cost_kernel<<<sh->B, kThreads, smem, st>>>(Lmax, S, kc, L, layers, (long long)layer_stride_B, strat, inst, time_s, mem_bytes, time_q,
+                                                   mem_q, trans_q, status);
+        if (tsmem > 48 * 1024) {                                   // long stacks or many strategies only; per device, so asked every time
+            cudaError_t e = cudaFuncSetAttribute(trans_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tsmem);
+            if (e != cudaSuccess) return e;
+        }
+        trans_kernel<<<tblocks, kThreads, tsmem, st>>>(sh->B, Lmax, S, L, layers, (long long)layer_stride_B, strat, inst, status, trans_q, ipc);
+        return cudaGetLastError();
+    }
+    if (tsmem > smem) smem = tsmem;                                   // one launch, two roles: the larger of their needs
+    if (smem > 48 * 1024) {                                   // long stacks or many strategies only; per device, so asked every time
+        cudaError_t e = cudaFuncSetAttribute(cost_trans_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    cost_trans_kernel<<<sh->B + tblocks, kThreads, smem, st>>>(sh->B, Lmax, S, kc, L, layers, (long long)layer_stride_B, strat, inst, time_s,
+                                                              mem_bytes, time_q, mem_q, trans_q, status, ipc);
     return cudaGetLastError();
 }
