@@ -100,3 +100,18 @@ def test_bad_descriptors_flag_the_instance_end_to_end(orc, galv):
     w2.strat["tp"][5] = 0
     sb2 = run_and_compare(orc, galv, w2, False)
     assert sb2.status.cpu().tolist() == [2, 2, 2]
+
+
+def test_large_batch_takes_two_kernels_and_small_batch_one(orc, galv):
+    """Past 1024 instances the layer tables and the transition matrices come from two launches (the second reads the
+    first's verdict on the descriptors); up to 1024 from one (the transition CTAs test the descriptors themselves).
+    Both must agree with the oracle, flagged instances included."""
+    strat = inputs.strategy_table((1, 2, 4, 8), (0, 3), (0, 1), (0, 1))
+    for B in (1024, 1100):
+        w = stack(90 + B, B, 9, strat, "alternate", per_instance=True, ragged=True)
+        w.inst["bw_tp"][B - 3] = -1.0                           # flagged by the instance parameters
+        w.layers["h"][B // 2, 0] = 0.0                          # flagged by a layer (every instance has at least one)
+        sb = run_and_compare(orc, galv, w, False)
+        st = sb.status.cpu().numpy()
+        assert st[B - 3] == 2 and st[B // 2] == 2 and (st != 0).sum() == 2
+        assert (sb.trans_q[B - 3].cpu().numpy() == -1).all() and (sb.trans_q[B // 2].cpu().numpy() == -1).all()
