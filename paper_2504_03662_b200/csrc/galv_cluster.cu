@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(416, 1) cluster_search_kernel(const ClArgs a, 
         i = s_inst;
     }
 
-    // ---- validation (every CTA of the cluster comes to the same verdict: nobody is left waiting at a barrier)
+    // ---- validation (every CTA of the cluster comes to the same result: nobody is left waiting at a barrier)
     if (tid == 0) { s_sum = 0; s_tmax = 0; s_bad = 0; }
     __syncthreads();
     const int Li = a.L[i];

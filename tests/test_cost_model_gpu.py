@@ -104,7 +104,7 @@ def test_bad_descriptors_flag_the_instance_end_to_end(orc, galv):
 
 def test_large_batch_takes_two_kernels_and_small_batch_one(orc, galv):
     """Past 1024 instances the layer tables and the transition matrices come from two launches (the second reads the
-    first's verdict on the descriptors); up to 1024 from one (the transition CTAs test the descriptors themselves).
+    first's status word for each instance); up to 1024 from one (the transition CTAs test the descriptors themselves).
     Both must agree with the oracle, flagged instances included."""
     strat = inputs.strategy_table((1, 2, 4, 8), (0, 3), (0, 1), (0, 1))
     for B in (1024, 1100):

@@ -745,7 +745,7 @@ def test_cluster_kernel_more_instances_than_cluster_slots(orc, galv):
 
 
 def test_cluster_kernel_flagged_instances(orc, galv):
-    """Validation inside the cluster kernel: the same verdicts as the validation pass of the tiled path."""
+    """Validation inside the cluster kernel: the same status bits as the validation pass of the tiled path."""
     from paper_2504_03662_b200 import binding as gb
     w = inputs.random_tables(5, 6, 4, 6, 50, ragged=True)
     w.time_q[1, 0, 2] = -7
