@@ -261,22 +261,41 @@ __device__ __forceinline__ void trans_body(const int cta, unsigned char* smem_ra
     for (int s = tid; s < S; s += kThreads)
         if (slot[s] < 0) slot[s] = slot[-slot[s] - 1];                    // the others copy it (an opener's entry is final by now)
     const bool vec = (S & 3) == 0;
-    for (int n = 0; n < inst_per_cta; ++n) {
-        const int i = cta * inst_per_cta + n;
-        if (i >= B) break;
-        __syncthreads();                                        // classes known; the last instance's table is no longer read
-        const int Li = L[i];
-        if (Li < 1 || Li > Lmax) continue;                      // out of range: nothing written
-        if (status && status[i] != 0) continue;                 // bad descriptor: already -1
-        const galv_layer_desc ly = layers[(long long)i * layer_stride_B];
-        const galv_inst_params in = inst[i];
-        if (!status) {
-            int bad = s_sbad | (inst_ok(in) ? 0 : 1);
-            for (int l = tid; l < Li; l += kThreads) bad |= layer_ok(layers[(long long)i * layer_stride_B + l]) ? 0 : 1;
-            if (__syncthreads_or(bad)) continue;                // flagged: the cost role writes -1 into this matrix too
+    __syncthreads();                                            // classes known
+    // As many instances at a time as their pair tables fit into the table's room (S * S words; at most S classes):
+    // one round of evaluations, one barrier, one run of stores for all of them.
+    __shared__ int s_ok[8];
+    const int nn = ncls * ncls;
+    const int cap = max(1, min(8, (S * S) / max(1, nn)));
+    for (int n0 = 0; n0 < inst_per_cta; n0 += cap) {
+        const int g = min(cap, inst_per_cta - n0);
+        __syncthreads();                                        // the last group's tables are no longer read
+        for (int n = 0; n < g; ++n) {
+            const int i = cta * inst_per_cta + n0 + n;
+            int ok = 0;
+            if (i < B) {
+                const int Li = L[i];
+                ok = Li >= 1 && Li <= Lmax;                     // out of range: nothing written
+                if (ok && status) ok = status[i] == 0;          // bad descriptor: already -1
+                if (!status) {
+                    int bad = 0;
+                    if (ok) {
+                        bad = s_sbad | (inst_ok(inst[i]) ? 0 : 1);
+                        for (int l = tid; l < Li; l += kThreads) bad |= layer_ok(layers[(long long)i * layer_stride_B + l]) ? 0 : 1;
+                    }
+                    if (__syncthreads_or(bad)) ok = 0;          // flagged: the cost role writes -1 into this matrix too
+                }
+            }
+            if (tid == 0) s_ok[n] = ok;
         }
-        for (int e = tid; e < ncls * ncls; e += kThreads) {
-            const int ka = e / ncls, kc = e - ka * ncls;
+        __syncthreads();
+        for (int e = tid; e < g * nn; e += kThreads) {
+            const int n = e / nn, r = e - n * nn;
+            if (!s_ok[n]) continue;
+            const int i = cta * inst_per_cta + n0 + n;
+            const galv_layer_desc ly = layers[(long long)i * layer_stride_B];
+            const galv_inst_params in = inst[i];
+            const int ka = r / ncls, kc = r - ka * ncls;
             const galv_strategy_desc sa = strat[rep[ka]], sc = strat[rep[kc]];
             const double bq = in.b / sc.batch_div;
             const double bytes = bq * ly.seq * ly.h * in.bytes_per_elem;
@@ -284,17 +303,22 @@ __device__ __forceinline__ void trans_body(const int cta, unsigned char* smem_ra
             tab[e] = quant_time(t, in.time_unit_ns);
         }
         __syncthreads();
-        int32_t* const out = trans_q + (size_t)i * S * S;
-        if (vec) {
-            for (int e = tid; e < S * S / 4; e += kThreads) {
-                const int a = (4 * e) / S, c = 4 * e - a * S;
-                const int32_t* row = tab + slot[a] * ncls;
-                reinterpret_cast<int4*>(out)[e] = make_int4(row[slot[c]], row[slot[c + 1]], row[slot[c + 2]], row[slot[c + 3]]);
-            }
-        } else {
-            for (int e = tid; e < S * S; e += kThreads) {
-                const int a = e / S, c = e - a * S;
-                out[e] = tab[slot[a] * ncls + slot[c]];
+        for (int n = 0; n < g; ++n) {
+            if (!s_ok[n]) continue;
+            const int i = cta * inst_per_cta + n0 + n;
+            int32_t* const out = trans_q + (size_t)i * S * S;
+            const int32_t* const tb = tab + n * nn;
+            if (vec) {
+                for (int e = tid; e < S * S / 4; e += kThreads) {
+                    const int a = (4 * e) / S, c = 4 * e - a * S;
+                    const int32_t* row = tb + slot[a] * ncls;
+                    reinterpret_cast<int4*>(out)[e] = make_int4(row[slot[c]], row[slot[c + 1]], row[slot[c + 2]], row[slot[c + 3]]);
+                }
+            } else {
+                for (int e = tid; e < S * S; e += kThreads) {
+                    const int a = e / S, c = e - a * S;
+                    out[e] = tb[slot[a] * ncls + slot[c]];
+                }
             }
         }
     }
