@@ -152,6 +152,7 @@ __global__ void __launch_bounds__(416, 1) cluster_search_kernel(const ClArgs a, 
     int* const fillc = reinterpret_cast<int*>(rows + 2 * nrec);                            // [2][SP8] leading cells of each row to fill with +inf
     int* const fillmax = fillc + 2 * SP8;                                                  // [2] the largest of them (padded to 4 ints)
     int32_t* const dump = fillmax + 4;                                                     // [32 * TM] where stores of skipped strategies go
+    int* const cdelta = dump + 32 * TM;                                                    // [16] cluster-window address of CTA d minus this CTA's own shared address
 
     if (blockIdx.x == 0 && tid == 0) { a.path[0] = 0; a.path[3] = 2; }      // no error flag to raise; the cluster kernel ran
 
@@ -260,6 +261,9 @@ __global__ void __launch_bounds__(416, 1) cluster_search_kernel(const ClArgs a, 
         prepare_layer(warp, m0, t0);
     }
     for (int x = tid; x < 32 * TM; x += NT) dump[x] = 0;
+    // where the other CTAs' buffers lie in the cluster window: asked once, not once per store (the mapping is an
+    // offset per CTA; asking inside the push puts its latency on every strategy's chain of branches)
+    if (tid < 16) cdelta[tid] = (int)(map_to_rank(smem_addr(buf0), (uint32_t)min(tid, CL - 1)) - smem_addr(buf0));
     {
         const int32_t* T = T0 + (a.trans_layer ? a.trans_layer : 0);       // matrix 1 is paid between layers 0 and 1
         int32_t* dst = tsm + (a.trans_layer ? tmat : 0);                    // per layer: matrix l sits in tsm[l & 1]
@@ -395,42 +399,24 @@ __global__ void __launch_bounds__(416, 1) cluster_search_kernel(const ClArgs a, 
                         for (int j = 0; j < TM; ++j) y[j * 32] = __viaddmin_s32(acc[j][u], r[u].z, kInf);    // +inf stays +inf
                     }
                 } else {
+                    // Some strategy's tile leaves the CTA or straddles two: the whole unit goes through the cluster window
+                    // (what stays at home too), one predicated store a register and no branch - a chain of branches per
+                    // strategy cost the warps that own such tiles three times the time of the stores themselves.
+                    // A whole tile has w = the largest int: its columns pass the test against w and lie below W.
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
-                        if (r[u].x < 0) continue;                           // nothing of this tile lands inside the budget
-                        const bool home = r[u].x == rank;
+                        const int dx = r[u].x < 0 ? 0 : r[u].x;
                         const uint32_t row = ybase + (uint32_t)((sg * 8 + u) * W) * 4u;
-                        int32_t* const y = yl + u * W + r[u].y;
-                        if (r[u].w == kWholeTile) {
-                            // all of it in one CTA's columns
-                            const uint32_t ra = home ? 0u : map_to_rank(row + (uint32_t)(r[u].y + lane) * 4u, (uint32_t)r[u].x);
+                        const uint32_t ra0 = row + (uint32_t)cdelta[dx];
+                        const uint32_t ra1 = row + (uint32_t)cdelta[min(dx + 1, CL - 1)] - (uint32_t)W * 4u;
+                        const bool lands = r[u].x >= 0;
 #pragma unroll
-                            for (int j = 0; j < TM; ++j)
-                                if (j < nj) {
-                                    const int v = __viaddmin_s32(acc[j][u], r[u].z, kInf);
-                                    if (home) y[j * 32] = v;
-                                    else st_cluster(ra + j * 128u, v);
-                                }
-                        } else {
-                            // the tile straddles two CTAs or the edge of the budget: every column is checked.  What stays
-                            // at home goes by plain stores; only what crosses to another CTA takes the cluster window.
-                            const uint32_t ra0 = home ? 0u : map_to_rank(row, (uint32_t)r[u].x);
-                            const uint32_t ra1 = map_to_rank(row, (uint32_t)min(r[u].x + 1, CL - 1)) - (uint32_t)W * 4u;
-#pragma unroll
-                            for (int j = 0; j < TM; ++j)
-                                if (j < nj) {
-                                    const int x = r[u].y + j * 32 + lane;
-                                    const int v = __viaddmin_s32(acc[j][u], r[u].z, kInf);
-                                    if (x <= r[u].w) {
-                                        if (x < W) {
-                                            if (home) y[j * 32] = v;
-                                            else st_cluster(ra0 + (uint32_t)x * 4u, v);
-                                        } else {
-                                            st_cluster(ra1 + (uint32_t)x * 4u, v);
-                                        }
-                                    }
-                                }
-                        }
+                        for (int j = 0; j < TM; ++j)
+                            if (j < nj) {
+                                const int x = r[u].y + j * 32 + lane;
+                                const int v = __viaddmin_s32(acc[j][u], r[u].z, kInf);
+                                if (lands && x <= r[u].w) st_cluster((x < W ? ra0 : ra1) + (uint32_t)x * 4u, v);
+                            }
                     }
                 }
             }
@@ -578,7 +564,7 @@ bool galv_cluster_plan(const galv_ctx* ctx, const galv_shape* sh, ClPlan* out)
         if (want_cl && cl != want_cl) continue;
         const int g = (Gt + cl - 1) / cl;
         if (cl > 1 && (g < 3 || g * (cl - 1) >= Gt)) continue;
-        const long long smem = (long long)2 * S * g * 32 * 4 + (long long)nT * S * sp8 * 4 + (long long)2 * ((g + 1) / 2) * sp8 * 16 + (long long)2 * sp8 * 4 + 16 + 512;
+        const long long smem = (long long)2 * S * g * 32 * 4 + (long long)nT * S * sp8 * 4 + (long long)2 * ((g + 1) / 2) * sp8 * 16 + (long long)2 * sp8 * 4 + 16 + 512 + 64;
         if (smem > budget) break;                            // smaller clusters need more per CTA
         ClPlan p;
         std::memset(&p, 0, sizeof(p));
