@@ -22,6 +22,8 @@ __device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v)
     return v;
 }
 
+// NJ: strategies per lane (S <= 32 * NJ): the walk's chain of selects, loads and ballots is as long as it has to be.
+template <int NJ>
 __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, long long trans_inst, long long trans_layer,
                                  const int32_t* __restrict__ L, const int32_t* __restrict__ time_q,
                                  const int32_t* __restrict__ mem_q, const int32_t* __restrict__ trans_q,
@@ -81,9 +83,9 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, lon
     // candidate of the step before), and the mem / time rows of the next layer down are fetched, whole,
     // while this layer's candidates are in flight; lane k%32 keeps entries k, k+32, ... (S <= 256).
     int cur = opt;                                             // C[l][m][s] of the cell the walk stands on
-    int mrow[8], trow[8];
+    int mrow[NJ], trow[NJ];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < NJ; ++j) {
         const int k = lane + 32 * j;
         mrow[j] = k < S ? mq[(Li - 1) * S + k] : 0;
         trow[j] = k < S ? tq[(Li - 1) * S + k] : 0;
@@ -92,7 +94,7 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, lon
         if (lane == 0) pl[l] = s;
         int msel = mrow[0], tsel = trow[0];
 #pragma unroll
-        for (int j = 1; j < 8; ++j) {
+        for (int j = 1; j < NJ; ++j) {
             msel = (s >> 5) == j ? mrow[j] : msel;
             tsel = (s >> 5) == j ? trow[j] : tsel;
         }
@@ -105,7 +107,7 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, lon
         }
         if (l == 0) break;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {                          // rows of layer l-1, needed one step from now
+        for (int j = 0; j < NJ; ++j) {                          // rows of layer l-1, needed one step from now
             const int k = lane + 32 * j;
             mrow[j] = k < S ? mq[(l - 1) * S + k] : 0;
             trow[j] = k < S ? tq[(l - 1) * S + k] : 0;
@@ -119,15 +121,15 @@ __global__ void backtrack_kernel(int B, int Lmax, int S, int M, int m_pitch, lon
             const int32_t* T = T0 + (size_t)l * trans_layer;       // paid between layers l-1 and l
             sp = 255;
             // every row's candidate is asked for before the first is looked at: one round trip to memory, not one per 32 rows
-            int cv[8], tv[8];
+            int cv[NJ], tv[NJ];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < NJ; ++j) {
                 const int k = lane + 32 * j;
                 cv[j] = k < S ? prev[(size_t)k * m_pitch] : kInf;
                 tv[j] = k < S ? T[k * S + s] : 0;
             }
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < NJ; ++j) {
                 if (32 * j >= S) break;
                 const bool hit = (cv[j] < kInf) && (cv[j] + tv[j] == target);
                 const unsigned b = __ballot_sync(0xffffffffu, hit);
@@ -158,8 +160,14 @@ cudaError_t galv_backtrack_launch(const galv_shape* sh, const int32_t* L, const 
                                   cudaStream_t st)
 {
     const int warps = 4;
-    backtrack_kernel<<<(sh->B + warps - 1) / warps, warps * 32, 0, st>>>(
-        sh->B, sh->Lmax, sh->S, sh->M, sh->m_pitch, galv_trans_inst(sh), galv_trans_layer(sh), L, time_q, mem_q, trans_q, C, A, C_last, budget,
-        opt_cost, plan, mem_used, status);
+    const dim3 grid((sh->B + warps - 1) / warps), block(warps * 32);
+#define GALV_WALK(NJ) backtrack_kernel<NJ><<<grid, block, 0, st>>>( \
+        sh->B, sh->Lmax, sh->S, sh->M, sh->m_pitch, galv_trans_inst(sh), galv_trans_layer(sh), L, time_q, mem_q, trans_q, C, A, C_last, budget, \
+        opt_cost, plan, mem_used, status)
+    if (sh->S <= 32) GALV_WALK(1);
+    else if (sh->S <= 64) GALV_WALK(2);
+    else if (sh->S <= 128) GALV_WALK(4);
+    else GALV_WALK(8);
+#undef GALV_WALK
     return cudaGetLastError();
 }
